@@ -1,0 +1,315 @@
+// LU-KV prefill compression path -- CPU ORACLE (test infrastructure, not product code).
+//
+// A plain, slow, single-threaded restatement of what the path computes, in double
+// precision, written from the paper's definitions and used only to check the CUDA
+// library: the tests, the smoke check and the benchmark's CPU-baseline leg call it.
+// It shares no code, header, table or helper with the CUDA path and must never be
+// reached from the product path.
+//
+// Stages (each function cites the passage it follows):
+//   score    : SnapKV-style observation-window proxy. Attention weights are the
+//              scaled-dot-product softmax of Eq. 1 (Sec. 3.1) with scale 1/sqrt(d_h);
+//              the paper only names the proxy ("accumulated attention scores over an
+//              observation window", Sec. 5.1; kernel 7 / window 32 in the baseline
+//              hyper-parameter table), so the window/causal/sum/pool reading is the
+//              conventional SnapKV one and is listed in the design notes.
+//   hull     : PAVA projection of the marginal decreases onto a non-negative,
+//              non-increasing sequence (Sec. 4.2, Eq. "marginal_gain"; App. A.2).
+//   allocate : marginal-utility greedy == the B largest gains under the per-head prefix
+//              constraint (Sec. 4.2 relaxed objective; App. A.2 "Optimality of greedy").
+//   select   : top-b positions of a head by the proxy (Sec. 4.3 "Eviction"; M^pi(k) of
+//              Sec. 3.2), ties by lower index (App. A.1 allows any fixed rule).
+//   gather   : the retained index set I of Sec. 3.2 materialised as a packed cache.
+//
+// Pins (see tests, "-m not gpu"): softmax rows sum to one; closed form for identical
+// keys; single-row case against a library softmax; pooling against a library max filter;
+// PAVA against a library isotonic regression, a monotone-chain hull and the O(P^2)
+// majorant definition; greedy against exhaustive search; selection against a full sort;
+// uniform budgets against a library-op SnapKV; gather by byte equality.
+// No function here is "parity unpinned".
+//
+// Build: g++ -O2 -std=c++17 -ffp-contract=off -shared -fPIC lukv_oracle.cpp -o liblukv_oracle.so
+
+#include <algorithm>
+#include <cfloat>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <numeric>
+#include <vector>
+
+namespace {
+
+// bf16 is the upper half of an IEEE binary32: widening is exact.
+inline float bf16_bits_to_float(uint16_t b) {
+  uint32_t u = static_cast<uint32_t>(b) << 16;
+  float f;
+  std::memcpy(&f, &u, sizeof f);
+  return f;
+}
+
+// dtype 0: bf16 stored as uint16 bit patterns; dtype 1: fp32.
+inline double load_elem(const void* base, int dtype, int64_t idx) {
+  if (dtype == 0) return static_cast<double>(bf16_bits_to_float(static_cast<const uint16_t*>(base)[idx]));
+  return static_cast<double>(static_cast<const float*>(base)[idx]);
+}
+
+inline size_t elem_size(int dtype) { return dtype == 0 ? 2 : 4; }
+
+// Round a double to fp32 (nearest-even); magnitudes below FLT_MIN become +0, mirroring
+// the flush-to-zero arithmetic of the device the oracle is compared with.
+inline float to_f32_ftz(double x) {
+  float f = static_cast<float>(x);
+  if (std::fabs(f) < FLT_MIN) f = 0.0f;
+  return f;
+}
+
+struct Dims {
+  int S, L, H, G, d, T, w, kp, dtype, P;
+  double scale;
+  int N() const { return L * H; }
+  int n() const { return T - w; }
+};
+
+// ---- score ---------------------------------------------------------------------------
+// One KV head. q_head: [G][w][d] (the G query heads of this KV head are contiguous in
+// the [H*G] axis), k_head: [T][d].
+// Row r=(g,i) is the query at position n+i; it sees keys j <= n+i (causal, Eq. 1 applied
+// at that position).  prob (optional): [G*w][T], masked entries 0.  raw_full (optional):
+// [T] column sums over all rows, in double.
+void score_head(const void* q_head, const void* k_head, int dtype, int G, int w, int d, int T,
+                double scale, double* prob, double* raw_full) {
+  const int n = T - w;
+  std::vector<double> kd(static_cast<size_t>(T) * d);
+  for (int64_t e = 0; e < static_cast<int64_t>(T) * d; ++e) kd[e] = load_elem(k_head, dtype, e);
+  std::vector<double> qd(d), x(T);
+  if (raw_full) std::fill(raw_full, raw_full + T, 0.0);
+  for (int g = 0; g < G; ++g) {
+    for (int i = 0; i < w; ++i) {
+      const int r = g * w + i;
+      for (int c = 0; c < d; ++c) qd[c] = load_elem(q_head, dtype, (static_cast<int64_t>(g) * w + i) * d + c);
+      const int visible = n + i + 1;  // keys 0 .. n+i
+      double m = -INFINITY;
+      for (int j = 0; j < visible; ++j) {
+        double acc = 0.0;
+        const double* kj = &kd[static_cast<size_t>(j) * d];
+        for (int c = 0; c < d; ++c) acc += qd[c] * kj[c];
+        x[j] = scale * acc;
+        if (x[j] > m) m = x[j];
+      }
+      double Z = 0.0;
+      for (int j = 0; j < visible; ++j) Z += std::exp(x[j] - m);
+      for (int j = 0; j < visible; ++j) {
+        const double p = std::exp(x[j] - m) / Z;
+        if (prob) prob[static_cast<size_t>(r) * T + j] = p;
+        if (raw_full) raw_full[j] += p;
+      }
+      if (prob)
+        for (int j = visible; j < T; ++j) prob[static_cast<size_t>(r) * T + j] = 0.0;
+    }
+  }
+}
+
+// Centred, stride-1 max filter of odd width kp over [0,n); the filter window is clipped
+// at both ends (equivalently padded with -inf).
+void max_pool(const double* raw, int n, int kp, double* pooled) {
+  const int half = kp / 2;
+  for (int j = 0; j < n; ++j) {
+    const int lo = std::max(0, j - half), hi = std::min(n - 1, j + half);
+    double best = raw[lo];
+    for (int t = lo + 1; t <= hi; ++t) best = std::max(best, raw[t]);
+    pooled[j] = best;
+  }
+}
+
+// ---- hull ----------------------------------------------------------------------------
+// PAVA on the P-1 increments of a utility curve U[0..P-1] (utility = L(0) - L(b), so its
+// increments are the paper's marginal decreases of the loss).  Blocks are kept on a
+// stack as [l, r) spans of curve points; a block's value is its mean increment
+// (U[r]-U[l])/(r-l).  A new increment is pushed as its own block and merged with the
+// block before it while that block's mean is <= the new one's (violating or tying the
+// required non-increasing order).  Each segment's gain is its block mean clipped at 0.
+void pava_gains(const float* U, int P, double* gains) {
+  struct Block { int l, r; double mean; };
+  std::vector<Block> st;
+  st.reserve(P);
+  for (int k = 0; k + 1 < P; ++k) {
+    Block cur{k, k + 1, (static_cast<double>(U[k + 1]) - static_cast<double>(U[k])) / 1.0};
+    while (!st.empty() && st.back().mean <= cur.mean) {
+      cur.l = st.back().l;
+      st.pop_back();
+      cur.mean = (static_cast<double>(U[cur.r]) - static_cast<double>(U[cur.l])) / static_cast<double>(cur.r - cur.l);
+    }
+    st.push_back(cur);
+  }
+  for (const Block& b : st) {
+    const double g = b.mean > 0.0 ? b.mean : 0.0;
+    for (int k = b.l; k < b.r; ++k) gains[k] = g;
+  }
+}
+
+// Capacity (tokens) of segment k of a head: the curve grid has step s = T/(P-1) tokens
+// and only the n = T - w non-window positions can be bought.
+inline int64_t seg_cap(int k, int64_t s, int64_t n) {
+  int64_t c = n - static_cast<int64_t>(k) * s;
+  if (c < 0) c = 0;
+  if (c > s) c = s;
+  return c;
+}
+
+struct Item { float gain; int k; int hid; int64_t cap; };
+
+// ---- select --------------------------------------------------------------------------
+// First b positions of the order (score descending, index ascending), emitted ascending.
+void select_head(const float* pooled, int n, int b, int32_t* kept) {
+  std::vector<int32_t> order(n);
+  std::iota(order.begin(), order.end(), 0);
+  std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t c) { return pooled[a] > pooled[c]; });
+  std::vector<int32_t> top(order.begin(), order.begin() + b);
+  std::sort(top.begin(), top.end());
+  std::copy(top.begin(), top.end(), kept);
+}
+
+}  // namespace
+
+extern "C" {
+
+// Probability matrix of one head (for the row-sum pin). prob: [G*w][T] doubles.
+void oracle_window_softmax(const void* q_head, const void* k_head, int dtype, int G, int w, int d, int T,
+                           float scale, double* prob) {
+  const double sc = scale != 0.0f ? static_cast<double>(scale) : 1.0 / std::sqrt(static_cast<double>(d));
+  score_head(q_head, k_head, dtype, G, w, d, T, sc, prob, nullptr);
+}
+
+// One head: raw_full [T] doubles (may be null), pooled [n] floats (may be null).
+void oracle_score_head(const void* q_head, const void* k_head, int dtype, int G, int w, int d, int T, int kp,
+                       float scale, double* raw_full, float* pooled) {
+  const double sc = scale != 0.0f ? static_cast<double>(scale) : 1.0 / std::sqrt(static_cast<double>(d));
+  const int n = T - w;
+  std::vector<double> raw(T), pl(n);
+  score_head(q_head, k_head, dtype, G, w, d, T, sc, nullptr, raw.data());
+  if (raw_full) std::copy(raw.begin(), raw.end(), raw_full);
+  if (pooled) {
+    max_pool(raw.data(), n, kp, pl.data());
+    for (int j = 0; j < n; ++j) pooled[j] = to_f32_ftz(pl[j]);
+  }
+}
+
+// All heads. q: [S][L][H*G][w][d], k: [S][L][H][T][d], scores: [S][L*H][n].
+void oracle_score(const void* q, const void* k, int dtype, int S, int L, int H, int G, int d, int T, int w,
+                  int kp, float scale, float* scores) {
+  const int n = T - w;
+  const size_t es = elem_size(dtype);
+  for (int64_t u = 0; u < static_cast<int64_t>(S) * L * H; ++u) {
+    const char* qh = static_cast<const char*>(q) + static_cast<size_t>(u) * G * w * d * es;
+    const char* kh = static_cast<const char*>(k) + static_cast<size_t>(u) * T * d * es;
+    oracle_score_head(qh, kh, dtype, G, w, d, T, kp, scale, nullptr, scores + u * n);
+  }
+}
+
+// Stand-alone max-pool over [0,n) (pin: library max filter).
+void oracle_max_pool(const double* raw, int n, int kp, double* pooled) { max_pool(raw, n, kp, pooled); }
+
+// Hull gains of N curves. curves: [N][P] floats; gains_f64 (may be null): [N][P-1]
+// doubles before the final rounding; gains_f32 (may be null): rounded once to fp32.
+void oracle_hull(const float* curves, int N, int P, double* gains_f64, float* gains_f32) {
+  std::vector<double> g(P - 1);
+  for (int h = 0; h < N; ++h) {
+    pava_gains(curves + static_cast<size_t>(h) * P, P, g.data());
+    for (int k = 0; k + 1 < P; ++k) {
+      if (gains_f64) gains_f64[static_cast<size_t>(h) * (P - 1) + k] = g[k];
+      if (gains_f32) gains_f32[static_cast<size_t>(h) * (P - 1) + k] = static_cast<float>(g[k]);
+    }
+  }
+}
+
+// Greedy allocation. curves: [N][P]; budgets_in: [S] selectable tokens per sequence;
+// budgets: [S][N]; offsets: [S*N+1] = exclusive scan of (budget + w) in head order
+// u = q*N + hid.  Returns 0, or -1 when some B_q is outside [0, N*n].
+// Items are all (hid,k) with non-zero capacity, ordered by (gain descending, k ascending,
+// hid ascending); they are consumed in that order until B_q tokens are spent, the last
+// one partially.
+int oracle_allocate(const float* curves, int N, int P, int T, int w, int S, const int64_t* budgets_in,
+                    int32_t* budgets, int32_t* offsets) {
+  const int64_t n = T - w, s = T / (P - 1);
+  std::vector<float> g(static_cast<size_t>(N) * (P - 1));
+  oracle_hull(curves, N, P, nullptr, g.data());
+  std::vector<Item> items;
+  for (int hid = 0; hid < N; ++hid)
+    for (int k = 0; k + 1 < P; ++k) {
+      const int64_t cap = seg_cap(k, s, n);
+      if (cap > 0) items.push_back(Item{g[static_cast<size_t>(hid) * (P - 1) + k], k, hid, cap});
+    }
+  std::sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
+    if (a.gain != b.gain) return a.gain > b.gain;
+    if (a.k != b.k) return a.k < b.k;
+    return a.hid < b.hid;
+  });
+  int64_t running = 0;
+  offsets[0] = 0;
+  for (int q = 0; q < S; ++q) {
+    const int64_t B = budgets_in[q];
+    if (B < 0 || B > static_cast<int64_t>(N) * n) return -1;
+    std::vector<int64_t> b(N, 0);
+    int64_t left = B;
+    for (const Item& it : items) {
+      if (left == 0) break;
+      const int64_t take = std::min(left, it.cap);
+      b[it.hid] += take;
+      left -= take;
+    }
+    for (int hid = 0; hid < N; ++hid) {
+      budgets[static_cast<size_t>(q) * N + hid] = static_cast<int32_t>(b[hid]);
+      running += b[hid] + w;
+      offsets[static_cast<size_t>(q) * N + hid + 1] = static_cast<int32_t>(running);
+    }
+  }
+  return 0;
+}
+
+// Top-b of one head. pooled: [n]; kept: [b], ascending positions.
+void oracle_select(const float* pooled, int n, int b, int32_t* kept) { select_head(pooled, n, b, kept); }
+
+// Selection + gather for all heads. scores: [S*N][n]; budgets: [S*N]; offsets: [S*N+1];
+// k,v: [S*N][T][d]; k_out,v_out: [rows][d]; kept_idx: [rows].  For head u the packed rows
+// [off, off+b) hold the kept positions in ascending order and rows [off+b, off+b+w) hold
+// the window positions n..T-1.
+void oracle_select_gather(const float* scores, const int32_t* budgets, const int32_t* offsets, const void* k,
+                          const void* v, int dtype, int heads, int T, int w, int d, void* k_out, void* v_out,
+                          int32_t* kept_idx) {
+  const int n = T - w;
+  const size_t row = static_cast<size_t>(d) * elem_size(dtype);
+  for (int64_t u = 0; u < heads; ++u) {
+    const int b = budgets[u];
+    int32_t* kept = kept_idx + offsets[u];
+    select_head(scores + u * n, n, b, kept);
+    for (int i = 0; i < w; ++i) kept[b + i] = n + i;
+    for (int t = 0; t < b + w; ++t) {
+      const size_t src = (static_cast<size_t>(u) * T + kept[t]) * row;
+      const size_t dst = (static_cast<size_t>(offsets[u]) + t) * row;
+      std::memcpy(static_cast<char*>(k_out) + dst, static_cast<const char*>(k) + src, row);
+      std::memcpy(static_cast<char*>(v_out) + dst, static_cast<const char*>(v) + src, row);
+    }
+  }
+}
+
+// The whole path: allocate (hull + greedy) and score are independent; selection needs
+// both; gather follows.  scores_out (may be null): [S*N][n] pooled scores.
+int oracle_compress(const void* q, const void* k, const void* v, const float* curves, const int64_t* budgets_in,
+                    int dtype, int S, int L, int H, int G, int d, int T, int w, int kp, int P, float scale,
+                    void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets, int32_t* offsets,
+                    float* scores_out) {
+  const int N = L * H, n = T - w;
+  if (oracle_allocate(curves, N, P, T, w, S, budgets_in, budgets, offsets) != 0) return -1;
+  std::vector<float> local;
+  float* sc = scores_out;
+  if (!sc) {
+    local.resize(static_cast<size_t>(S) * N * n);
+    sc = local.data();
+  }
+  oracle_score(q, k, dtype, S, L, H, G, d, T, w, kp, scale, sc);
+  oracle_select_gather(sc, budgets, offsets, k, v, dtype, S * N, T, w, d, k_out, v_out, kept_idx);
+  return 0;
+}
+
+}  // extern "C"

@@ -1,0 +1,169 @@
+"""ctypes front end of the CPU oracle (test infrastructure, not product code).
+
+Loads ``liblukv_oracle.so`` (built from ``lukv_oracle.cpp`` by :func:`build`) and wraps
+its entry points for numpy arrays.  Only the tests, the smoke check and the benchmark's
+CPU-baseline leg may import this module; the CUDA library and its Python binding never do.
+
+bf16 tensors are passed as ``uint16`` bit patterns (``dtype=0``), fp32 as ``float32``
+(``dtype=1``).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "lukv_oracle.cpp")
+_LIB = os.path.join(_HERE, "liblukv_oracle.so")
+_lib = None
+
+BF16, FP32 = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no fused multiply-add contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-shared", "-fPIC", _SRC, "-o", _LIB]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.oracle_allocate.restype = ctypes.c_int
+        _lib.oracle_compress.restype = ctypes.c_int
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _dtype_code(a: np.ndarray) -> int:
+    if a.dtype == np.uint16:
+        return BF16
+    if a.dtype == np.float32:
+        return FP32
+    raise TypeError(f"oracle takes uint16 (bf16 bits) or float32, got {a.dtype}")
+
+
+def _c(a, dtype=None):
+    a = np.ascontiguousarray(a) if dtype is None else np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def window_softmax(q_head, k_head, scale: float = 0.0) -> np.ndarray:
+    """Probabilities of one head: q_head [G][w][d], k_head [T][d] -> [G*w][T] float64."""
+    q_head, k_head = _c(q_head), _c(k_head)
+    G, w, d = q_head.shape
+    T = k_head.shape[0]
+    prob = np.empty((G * w, T), np.float64)
+    lib().oracle_window_softmax(_p(q_head), _p(k_head), _dtype_code(k_head), G, w, d, T,
+                                ctypes.c_float(scale), _p(prob))
+    return prob
+
+
+def score_head(q_head, k_head, kp: int, scale: float = 0.0):
+    """One head -> (raw_full [T] float64, pooled [T-w] float32)."""
+    q_head, k_head = _c(q_head), _c(k_head)
+    G, w, d = q_head.shape
+    T = k_head.shape[0]
+    raw = np.empty(T, np.float64)
+    pooled = np.empty(T - w, np.float32)
+    lib().oracle_score_head(_p(q_head), _p(k_head), _dtype_code(k_head), G, w, d, T, kp,
+                            ctypes.c_float(scale), _p(raw), _p(pooled))
+    return raw, pooled
+
+
+def score(q, k, G: int, kp: int, scale: float = 0.0) -> np.ndarray:
+    """q [S][L][H*G][w][d], k [S][L][H][T][d] -> pooled scores [S][L*H][T-w] float32."""
+    q, k = _c(q), _c(k)
+    S, L, HG, w, d = q.shape
+    H, T = k.shape[2], k.shape[3]
+    assert HG == H * G
+    out = np.empty((S, L * H, T - w), np.float32)
+    lib().oracle_score(_p(q), _p(k), _dtype_code(k), S, L, H, G, d, T, w, kp, ctypes.c_float(scale), _p(out))
+    return out
+
+
+def max_pool(raw, kp: int) -> np.ndarray:
+    raw = _c(raw, np.float64)
+    out = np.empty_like(raw)
+    lib().oracle_max_pool(_p(raw), raw.shape[0], kp, _p(out))
+    return out
+
+
+def hull(curves):
+    """curves [N][P] float32 -> (gains float64 [N][P-1], gains rounded once to float32)."""
+    curves = _c(curves, np.float32)
+    N, P = curves.shape
+    g64 = np.empty((N, P - 1), np.float64)
+    g32 = np.empty((N, P - 1), np.float32)
+    lib().oracle_hull(_p(curves), N, P, _p(g64), _p(g32))
+    return g64, g32
+
+
+def allocate(curves, T: int, w: int, budgets_in):
+    """curves [N][P], budgets_in [S] -> (budgets int32 [S][N], offsets int32 [S*N+1])."""
+    curves = _c(curves, np.float32)
+    budgets_in = _c(budgets_in, np.int64)
+    N, P = curves.shape
+    S = budgets_in.shape[0]
+    budgets = np.empty((S, N), np.int32)
+    offsets = np.empty(S * N + 1, np.int32)
+    rc = lib().oracle_allocate(_p(curves), N, P, T, w, S, _p(budgets_in), _p(budgets), _p(offsets))
+    if rc != 0:
+        raise ValueError("budget outside [0, N*(T-w)]")
+    return budgets, offsets
+
+
+def select(pooled, b: int) -> np.ndarray:
+    pooled = _c(pooled, np.float32)
+    kept = np.empty(b, np.int32)
+    lib().oracle_select(_p(pooled), pooled.shape[0], b, _p(kept))
+    return kept
+
+
+def select_gather(scores, budgets, offsets, k, v, w: int):
+    """scores [U][n], budgets [U], offsets [U+1], k/v [U][T][d] -> (k_out, v_out, kept_idx)."""
+    scores = _c(scores, np.float32)
+    budgets = _c(budgets, np.int32).reshape(-1)
+    offsets = _c(offsets, np.int32)
+    k, v = _c(k), _c(v)
+    U = budgets.shape[0]
+    T, d = k.shape[-2], k.shape[-1]
+    rows = int(offsets[-1])
+    k_out = np.empty((rows, d), k.dtype)
+    v_out = np.empty((rows, d), v.dtype)
+    kept = np.empty(rows, np.int32)
+    lib().oracle_select_gather(_p(scores), _p(budgets), _p(offsets), _p(k), _p(v), _dtype_code(k), U, T, w, d,
+                               _p(k_out), _p(v_out), _p(kept))
+    return k_out, v_out, kept
+
+
+def compress(q, k, v, curves, budgets_in, G: int, kp: int, scale: float = 0.0):
+    """The whole path. Returns dict(k_out, v_out, kept_idx, budgets, offsets, scores)."""
+    q, k, v = _c(q), _c(k), _c(v)
+    curves = _c(curves, np.float32)
+    budgets_in = _c(budgets_in, np.int64)
+    S, L, HG, w, d = q.shape
+    H, T = k.shape[2], k.shape[3]
+    N, P = curves.shape
+    assert HG == H * G and N == L * H
+    rows = int(budgets_in.sum()) + S * N * w
+    out = dict(
+        k_out=np.empty((rows, d), k.dtype), v_out=np.empty((rows, d), v.dtype),
+        kept_idx=np.empty(rows, np.int32), budgets=np.empty((S, N), np.int32),
+        offsets=np.empty(S * N + 1, np.int32), scores=np.empty((S, N, T - w), np.float32))
+    rc = lib().oracle_compress(_p(q), _p(k), _p(v), _p(curves), _p(budgets_in), _dtype_code(k), S, L, H, G, d,
+                               T, w, kp, P, ctypes.c_float(scale), _p(out["k_out"]), _p(out["v_out"]),
+                               _p(out["kept_idx"]), _p(out["budgets"]), _p(out["offsets"]), _p(out["scores"]))
+    if rc != 0:
+        raise ValueError("budget outside [0, N*(T-w)]")
+    return out
