@@ -52,7 +52,7 @@ def test_curves_and_budgets():
     assert np.all(inc > 0) and abs(inc.mean() - 1.4) < 0.05        # E = 0.8*1 + 0.2*3
     assert np.any(np.diff(inc, axis=1) > 0)                         # non-concave
     cc = synth.gen_curves(wl, concave=True)
-    assert np.all(np.diff(np.diff(cc.astype(np.float64), axis=1), axis=1) <= 1e-5)
+    assert np.all(np.diff(np.diff(cc.astype(np.float64), axis=1), axis=1) <= 2e-4)      # up to fp32 rounding of the sums
     assert wl.budgets().tolist() == [1677721] and wl.total_rows() == 1685913
     w4 = synth.CONFIGS["batch8_16k_mixed"]
     assert w4.budgets().tolist() == [419430, 2097152] * 4 and w4.total_rows() == 10197400
