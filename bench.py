@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the fused LU-KV compression path (score + allocate + select + gather).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One "step" is one lukv_compress call over one batch of seeded synthetic input.  The default
+workload is the Llama-3.1-8B shaped full model at 32k context (256 KV heads allocated
+jointly, bf16).  Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank compresses
+its own copy of the workload (sequences are independent: weak scaling, no data-path
+collective) and the time is the max over ranks.
+
+--impl reference times the CPU oracle (as it stands, single thread) on a bounded sample of
+heads of the same workload and prints the same line with "impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "KV-compress context tokens/s (score+allocate+select+gather)"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b_32k")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-heads", type=int, default=24, help="heads in the CPU-baseline sample")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+# ---- CPU oracle leg (cpu_baseline of our arm, and the whole reference arm) --------------------
+
+def oracle_sample_seconds(wl, heads):
+    """Seconds the oracle needs for allocation (all heads) plus score/select/gather of `heads`
+    sampled heads; returns (seconds, seconds extrapolated to the whole workload)."""
+    import numpy as np
+    from oracle import lukv_oracle as O
+    from paper_2602_08585_b200 import synth
+    curves = synth.gen_curves(wl)
+    Bs = wl.budgets()
+    total_heads = wl.S * wl.N
+    heads = min(heads, total_heads)
+    sample = [int(x) for x in np.linspace(0, total_heads - 1, heads).round()]
+    data = []
+    for u in sample:
+        q, rem = divmod(u, wl.N)
+        layer, h = divmod(rem, wl.H)
+        qh, kh, vh = synth.gen_head(wl, q, layer, h, "cpu")
+        data.append((u, synth.to_numpy_bits(qh), synth.to_numpy_bits(kh), synth.to_numpy_bits(vh)))
+    t0 = time.perf_counter()
+    budgets, offsets = O.allocate(curves, wl.T, wl.w, Bs)
+    t_alloc = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    for u, qh, kh, vh in data:
+        _, pooled = O.score_head(qh, kh, wl.kp)
+        b = np.array([budgets.reshape(-1)[u]], np.int32)
+        off = np.array([0, b[0] + wl.w], np.int32)
+        O.select_gather(pooled[None], b, off, kh[None], vh[None], wl.w)
+    t_heads = time.perf_counter() - t0
+    return t_alloc + t_heads, t_alloc + t_heads * total_heads / heads, heads
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import lukv_oracle as O
+    from paper_2602_08585_b200 import synth
+    O.build()
+    wl = synth.CONFIGS[args.workload]
+    heads = max(1, min(4, wl.S * wl.N))
+    for _ in range(args.warmup):
+        oracle_sample_seconds(wl, 1)
+    full = []
+    for _ in range(args.steps):
+        _, extrap, used = oracle_sample_seconds(wl, heads)
+        full.append(extrap)
+    sec = sum(full) / len(full)
+    value = wl.S * wl.T / sec
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded)",
+        "config": {"workload": wl.name, "S": wl.S, "heads": wl.N, "T": wl.T, "w": wl.w, "keep": list(wl.keep)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"{heads} of {wl.S * wl.N} heads per step (score+select+gather) plus the full "
+                                   "allocation, single thread, extrapolated to all heads"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---- clocks ------------------------------------------------------------------------------------
+
+class ClockSampler(threading.Thread):
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, device_index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception as e:  # NVML missing: the clocks object says so
+            self.err = repr(e)
+
+    def sample_once(self):
+        nv = self.nv
+        self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+        try:
+            mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+        except Exception:
+            mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+        for bit, name in self.REASONS.items():
+            if mask & bit:
+                self.reasons.add(name)
+
+    def run(self):
+        while self.ok and not self._halt.is_set():
+            self.sample_once()
+            time.sleep(0.005)
+
+    def stop(self):
+        self._halt.set()
+        if self.ok:
+            self.join()
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "note": "NVML unavailable"}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+# ---- our arm -------------------------------------------------------------------------------------
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def kernel_bytes(name, wl, rows):
+    """Algorithmic bytes one launch of a kernel must move (inputs read once + outputs written once)."""
+    es = 2 if wl.dtype == "bf16" else 4
+    heads = wl.S * wl.N
+    k_bytes = heads * wl.T * wl.d * es
+    q_bytes = heads * wl.G * wl.w * wl.d * es
+    score_bytes = heads * wl.n * 4
+    row = wl.d * es
+    if name.startswith("score") and "lse" not in name:
+        return k_bytes + q_bytes + (score_bytes if name.endswith("2") or "fused" in name else 0)
+    if name == "max_pool":
+        return 2 * score_bytes
+    if name == "select":
+        return score_bytes + rows * 4
+    if name == "gather":
+        return rows * (2 * row * 2 + 4)
+    return 0
+
+
+def load_traffic(kernel, workload):
+    """DRAM bytes per launch from a committed ncu capture, if one is recorded."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            return json.load(f).get(workload, {}).get(kernel)
+    except Exception:
+        return None
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2602_08585_b200 import lukv, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (the path has no CPU fallback)"
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    lukv.lib()
+
+    wl = synth.CONFIGS[args.workload]
+    p = lukv.make_params(wl.S, wl.L, wl.H, wl.G, wl.d, wl.T, wl.w, wl.kp, wl.dtype, wl.P)
+    q, k, v = synth.gen_tensors(wl, "cuda")
+    curves_np = synth.gen_curves(wl)
+    curves = torch.from_numpy(curves_np).cuda()
+    Bs = wl.budgets()
+    ws = lukv.alloc_workspace(p)
+    out = lukv.Outputs(p, Bs)
+
+    def step():
+        lukv.lukv_compress(p, q, k, v, curves, Bs, out.k_out, out.v_out, out.kept_idx, out.budgets, out.offsets,
+                           out.rows, out.dev_status, ws)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 0)):
+        step()
+    launches_per_step = lukv.lukv_last_launch_count()
+    barrier()
+    sampler = ClockSampler(local)
+    if sampler.ok:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    if sampler.ok and not sampler.samples:
+        sampler.sample_once()
+    sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        dist.barrier()
+    assert int(out.dev_status.item()) == 0
+    tokens = wl.S * wl.T * world
+    value = tokens / (ms * 1e-3)
+
+    # ---- per-kernel device times (events after every kernel), dominant kernel roofline
+    peak, peak_src = measured_peak()
+    acc = {}
+    reps = 3
+    for _ in range(reps):
+        for name, t_ms in lukv.lukv_compress_profile(p, q, k, v, curves, Bs, out.k_out, out.v_out, out.kept_idx,
+                                                     out.budgets, out.offsets, out.rows, out.dev_status, ws):
+            a = acc.setdefault(name, [0.0, 0])
+            a[0] += t_ms
+            a[1] += 1
+    kernels = {name: {"ms_per_launch": tot / cnt, "launches_per_step": cnt // reps} for name, (tot, cnt) in acc.items()}
+    total_kernel_ms = sum(kv["ms_per_launch"] * kv["launches_per_step"] for kv in kernels.values())
+    for kv in kernels.values():
+        kv["share"] = kv["ms_per_launch"] * kv["launches_per_step"] / total_kernel_ms
+    dom = max(kernels, key=lambda nm: kernels[nm]["ms_per_launch"] * kernels[nm]["launches_per_step"])
+    dom_bytes = kernel_bytes(dom, wl, out.rows)
+    dom_gbs = dom_bytes / (kernels[dom]["ms_per_launch"] * 1e-3) / 1e9
+    roofline = {"kernel": dom, "bound": "hbm", "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
+                "frac": dom_gbs / peak, "peak_source": peak_src, "algorithmic_bytes_per_launch": dom_bytes,
+                "traffic": load_traffic(dom, wl.name)}
+    es = 2 if wl.dtype == "bf16" else 4
+    path_bytes = wl.S * wl.N * wl.T * wl.d * es + 2 * out.rows * wl.d * es   # K read + kept K/V written
+    path_gbs = path_bytes / (ms * 1e-3) / 1e9
+    path_roofline = {"bytes_per_step": path_bytes, "achieved": path_gbs, "unit": "GB/s",
+                     "frac_of_measured_peak": path_gbs / peak, "frac_of_nominal_8TBs": path_gbs / NOMINAL_HBM_GBS}
+
+    # ---- end to end through the C ABI with host buffers (pinned): H2D inputs, compress, D2H results
+    e2e = None
+    if not args.no_e2e:
+        try:
+            host_in = [t.cpu().pin_memory() for t in (q, k, v, curves)]
+            dev_in = [q, k, v, curves]
+            outs = [out.k_out, out.v_out, out.kept_idx, out.budgets, out.offsets]
+            host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+
+            def e2e_step():
+                for d_, h_ in zip(dev_in, host_in):
+                    d_.copy_(h_, non_blocking=True)
+                step()
+                for h_, d_ in zip(host_out, outs):
+                    h_.copy_(d_, non_blocking=True)
+
+            e2e_step()
+            barrier()
+            e0.record()
+            for _ in range(args.e2e_steps):
+                e2e_step()
+            e1.record()
+            torch.cuda.synchronize()
+            e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
+            if dist is not None:
+                t = torch.tensor([e2e_ms], device="cuda")
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                e2e_ms = float(t.item())
+            e2e = {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms, "steps": args.e2e_steps,
+                   "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_in)),
+                   "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_out))}
+            del host_in, host_out
+        except Exception as ex:  # e.g. not enough pinned host memory
+            e2e = {"value": None, "unit": UNIT, "error": repr(ex)[:200]}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import lukv_oracle as O
+        O.build()
+        sec, extrap, used = oracle_sample_seconds(wl, args.cpu_heads)
+        cpu_baseline = {"value": wl.S * wl.T / extrap, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "seconds_for_sample": sec,
+                        "sample": f"{used} of {wl.S * wl.N} heads (score+select+gather) plus the full allocation, "
+                                  "single thread, extrapolated to all heads"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 in / f32 accumulate" if wl.dtype == "bf16" else "f32",
+            "data": "synthetic (seeded)",
+            "config": {"workload": wl.name, "S": wl.S, "layers": wl.L, "kv_heads": wl.H, "gqa_group": wl.G,
+                       "head_dim": wl.d, "T": wl.T, "w": wl.w, "pool": wl.kp, "curve_points": wl.P,
+                       "keep": list(wl.keep), "packed_rows": out.rows,
+                       "l2": "inputs (K+V %.2f GB) exceed the 126 MB L2; no explicit flush" %
+                             (2 * wl.S * wl.N * wl.T * wl.d * es / 1e9),
+                       "parallelism": "replicas (one full workload per GPU)" if world > 1 else "single GPU"},
+            "clocks": sampler.summary(), "roofline": roofline, "path_roofline": path_roofline, "kernels": kernels,
+            "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": launches_per_step * args.steps,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

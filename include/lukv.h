@@ -1,0 +1,179 @@
+/*
+ * lukv.h -- C ABI of the LU-KV prefill-time KV-cache compression path for NVIDIA B200
+ * (sm_100a).  Four stages, all executed by hand-written CUDA kernels inside liblukv.so:
+ *
+ *   score     proxy importance of every cached position, per KV head
+ *   allocate  split a global token budget over the heads (hull relaxation + greedy)
+ *   select    per-head top-b positions by score
+ *   gather    compact the kept K/V rows (plus the always-kept observation window)
+ *
+ * Problem statement implemented (paper Sec. 4.2 Eq. "combinatorial_optimization" and its
+ * relaxed form, Sec. 4.3 "Online Execution"): given per-head utility-versus-budget
+ * curves, a global budget and the prefill KV cache, produce integer per-head budgets b
+ * with sum(b) = B exactly and, for every head, the retained set M^pi(b) of its top-b
+ * positions under the proxy metric pi (SnapKV-style observation-window attention).
+ *
+ * Conventions
+ *   - Every pointer is DEVICE memory unless marked HOST.  The caller owns every buffer;
+ *     the library allocates nothing, keeps no state between calls and never synchronises
+ *     the stream.  All work is enqueued on `stream` (a cudaStream_t passed as void*).
+ *   - Tensors are contiguous, row-major, in the layouts written next to each argument.
+ *   - Notation: S sequences, L layers, H KV heads per layer, N = L*H heads per sequence,
+ *     G query heads per KV head, d head dim, T context length, w observation window,
+ *     n = T-w rankable positions, kp max-pool width, P curve points per head,
+ *     s = T/(P-1) tokens per curve segment.  Head index u = (q*L + l)*H + h; the head id
+ *     inside a sequence is hid = l*H + h.
+ *   - Return value: 0 (LUKV_OK) or a negative lukv_status.  Argument errors are detected
+ *     on the host before anything is launched.  Inputs are assumed finite.
+ */
+#ifndef LUKV_H_
+#define LUKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define LUKV_API __attribute__((visibility("default")))
+#else
+#define LUKV_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lukv_status {
+  LUKV_OK = 0,
+  LUKV_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, flags != 0           */
+  LUKV_ERR_UNSUPPORTED = -2,         /* d not in {64,128}, unknown dtype, even kp, (P-1) does  */
+                                     /* not divide T, G*w > 256, P > 4097, sizes beyond int32  */
+  LUKV_ERR_BUDGET = -3,              /* some B_q < 0 or B_q > N*n                              */
+  LUKV_ERR_WORKSPACE_TOO_SMALL = -4, /* ws_bytes < lukv_workspace_bytes()                      */
+  LUKV_ERR_OUTPUT_TOO_SMALL = -5,    /* rows_cap < sum_q B_q + S*N*w                           */
+  LUKV_ERR_CUDA = -6,                /* a launch failed; cudaGetLastError() is left set        */
+  LUKV_ERR_TIMEOUT = -7              /* written to *dev_status only: a bounded device wait ran */
+                                     /* out; outputs of that call are unspecified              */
+} lukv_status;
+
+enum { LUKV_DTYPE_BF16 = 0, LUKV_DTYPE_FP32 = 1 };
+
+typedef struct lukv_params {
+  int32_t batch;        /* S >= 1                                                             */
+  int32_t n_layers;     /* L >= 1                                                             */
+  int32_t n_kv_heads;   /* H >= 1                                                             */
+  int32_t gqa_group;    /* G >= 1, G*w <= 256                                                 */
+  int32_t head_dim;     /* d in {64, 128}                                                     */
+  int32_t ctx_len;      /* T                                                                  */
+  int32_t window;       /* w, 1 <= w < T                                                      */
+  int32_t pool_kernel;  /* kp, odd, >= 1                                                      */
+  int32_t dtype;        /* LUKV_DTYPE_BF16 or LUKV_DTYPE_FP32: element type of Q, K and V     */
+  int32_t curve_points; /* P, 2 <= P <= 4097, (P-1) divides T                                 */
+  float softmax_scale;  /* 0 selects 1/sqrt(d) (Eq. 1)                                        */
+  int32_t flags;        /* reserved, must be 0                                                */
+} lukv_params_t;
+
+/* Bytes of scratch that any of the calls below needs for these parameters (one size fits
+ * all four).  The scratch must be 256-byte aligned.  Contents need no initialisation and
+ * are undefined afterwards. */
+LUKV_API int lukv_workspace_bytes(const lukv_params_t* params, size_t* bytes /* HOST, out */);
+
+/*
+ * Stage (a): proxy scoring.  Attention weights follow Eq. 1 (Sec. 3.1): softmax of
+ * scale * <q, k>.  The proxy is the SnapKV observation-window score the paper adopts as
+ * pi_1 (Sec. 5.1; window 32 / kernel 7 in its hyper-parameter table): for KV head u, the
+ * queries are the last w positions of its G query heads; the query at position n+i sees
+ * keys 0..n+i (causal); each row is soft-maxed over its visible keys; the probabilities
+ * are summed over the w rows and the G query heads; the resulting vector over the n
+ * non-window positions is max-pooled (width kp, stride 1, centred, clipped at the ends).
+ *
+ *   q_win  [S][L][H*G][w][d]  the queries of the last w positions (query head h*G+g
+ *                             belongs to KV head h)
+ *   k      [S][L][H][T][d]
+ *   scores [S][N][n] fp32     out: pooled scores (>= 0)
+ */
+LUKV_API int lukv_score(const lukv_params_t* params, const void* q_win, const void* k, float* scores, void* ws,
+               size_t ws_bytes, void* stream);
+
+/*
+ * Stage (b): global head-level budget allocation (Sec. 4.2; App. A.2).
+ * (b1) Hull relaxation: the P-1 increments of each head's utility curve are projected by
+ *      pool-adjacent-violators onto a non-increasing sequence and clipped at 0
+ *      (Eq. "marginal_gain"), in fp64, each gain rounded once to fp32.  Utility is
+ *      U(b) = L(0) - L(b), so these are the paper's marginal decreases of the loss.
+ * (b2) Greedy: curve point k is the utility of keeping the top k*s non-window tokens; all
+ *      tokens of segment k share its gain, and the segment can hold
+ *      cap = clamp(n - k*s, 0, s) tokens.  Segments are consumed in the order
+ *      (gain descending, k ascending, hid ascending) until B_q tokens are spent, the last
+ *      one partially -- the B_q largest marginal gains under the per-head prefix
+ *      constraint.  sum_hid budgets[q][hid] == B_q exactly.
+ *
+ *   curves     [N][P] fp32          utility curves, shared by all sequences
+ *   budgets_in [S] int64, HOST      selectable tokens B_q per sequence, 0 <= B_q <= N*n
+ *                                   (window rows are kept on top of it)
+ *   budgets    [S][N] int32         out
+ *   offsets    [S*N+1] int32        out: exclusive scan of (budgets + w) over u; head u
+ *                                   owns packed rows [offsets[u], offsets[u+1])
+ */
+LUKV_API int lukv_allocate(const lukv_params_t* params, const float* curves, const int64_t* budgets_in, int32_t* budgets,
+                  int32_t* offsets, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Stages (c)+(d): per-head top-b selection (Sec. 4.3 "Eviction": keep M^pi(b), the first b
+ * positions when ranked by score descending; ties go to the lower position, the fixed
+ * deterministic rule App. A.1 asks for) and compaction of the retained set (Sec. 3.2).
+ * For head u with b = budgets[u] and o = offsets[u]:
+ *   kept_idx[o .. o+b)      the selected positions, ascending
+ *   kept_idx[o+b .. o+b+w)  the window positions n .. T-1
+ *   k_out / v_out row r     = k / v row kept_idx[r] of head u, copied bit for bit
+ *
+ *   scores   [S][N][n] fp32   pooled scores (non-negative, finite)
+ *   budgets  [S][N] int32, offsets [S*N+1] int32   as produced by lukv_allocate; the
+ *            caller guarantees 0 <= budgets <= n and offsets consistent with them
+ *   k, v     [S][L][H][T][d]
+ *   k_out, v_out [rows_cap][d], kept_idx [rows_cap] int32   out
+ *   rows_cap rows available in the outputs; total rows = sum_q B_q + S*N*w is known on
+ *            the host.  Rows at or beyond rows_cap are never written.
+ */
+LUKV_API int lukv_select_gather(const lukv_params_t* params, const float* scores, const int32_t* budgets,
+                       const int32_t* offsets, const void* k, const void* v, void* k_out, void* v_out,
+                       int32_t* kept_idx, int64_t rows_cap, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The whole path in one call: score, allocate, select, gather (Sec. 4.2-4.3), with the
+ * intermediate scores kept in the workspace.  Arguments as above.  Returns
+ * LUKV_ERR_OUTPUT_TOO_SMALL when rows_cap < sum_q B_q + S*N*w.
+ *   dev_status [1] int32, may be NULL: set to 0 by the call; a kernel that gives up on a
+ *   bounded wait stores LUKV_ERR_TIMEOUT there.
+ */
+LUKV_API int lukv_compress(const lukv_params_t* params, const void* q_win, const void* k, const void* v,
+                  const float* curves, const int64_t* budgets_in, void* k_out, void* v_out, int32_t* kept_idx,
+                  int32_t* budgets, int32_t* offsets, int64_t rows_cap, int32_t* dev_status, void* ws,
+                  size_t ws_bytes, void* stream);
+
+/*
+ * Profiling variant of lukv_compress (the paper has no counterpart): same arguments and
+ * results, but a CUDA event is recorded after every kernel and the call SYNCHRONISES the
+ * stream before returning the per-kernel device times.  Not for production use.
+ *   times [max_times] HOST, out: kernel name (static string) and milliseconds, in launch
+ *   order; n_times HOST, out: entries written.  1 <= max_times <= 64.
+ */
+typedef struct lukv_kernel_time {
+  const char* name;
+  float ms;
+} lukv_kernel_time_t;
+LUKV_API int lukv_compress_profile(const lukv_params_t* params, const void* q_win, const void* k, const void* v,
+                                   const float* curves, const int64_t* budgets_in, void* k_out, void* v_out,
+                                   int32_t* kept_idx, int32_t* budgets, int32_t* offsets, int64_t rows_cap,
+                                   int32_t* dev_status, void* ws, size_t ws_bytes, void* stream,
+                                   lukv_kernel_time_t* times, int max_times, int* n_times);
+
+/* Static description of a status code. */
+LUKV_API const char* lukv_strerror(int code);
+
+/* Number of kernels the last successful call on this thread enqueued (for accounting). */
+LUKV_API int lukv_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LUKV_H_ */

@@ -1,0 +1,254 @@
+// C ABI of liblukv.so: argument validation, workspace carve-up and stage sequencing.
+// Every step of the path runs in the kernels of this library; there is no host fallback.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace lukv {
+
+static thread_local int g_last_launches = 0;
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+Workspace carve_workspace(const Dims& dm, void* base) {
+  Workspace ws;
+  char* p = static_cast<char*>(base);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    void* r = p ? p + off : nullptr;
+    off += align256(bytes);
+    return r;
+  };
+  const size_t heads = (size_t)dm.heads();
+  ws.raw = static_cast<float*>(take(heads * dm.n * sizeof(float)));
+  ws.pooled = static_cast<float*>(take(heads * dm.n * sizeof(float)));
+  ws.stats = static_cast<float*>(take(heads * score_chunks(dm) * dm.M * 2 * sizeof(float)));
+  ws.lse = static_cast<float*>(take(heads * dm.M * sizeof(float)));
+  ws.gains = static_cast<float*>(take((size_t)dm.N * (dm.P - 1) * sizeof(float)));
+  ws.bytes = off;
+  return ws;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Validates the parameter block and fills Dims.
+static int make_dims(const lukv_params_t* p, Dims* dm) {
+  if (!p) return LUKV_ERR_INVALID_ARG;
+  if (p->flags != 0) return LUKV_ERR_INVALID_ARG;
+  if (p->batch < 1 || p->n_layers < 1 || p->n_kv_heads < 1 || p->gqa_group < 1 || p->ctx_len < 2 || p->window < 1 ||
+      p->window >= p->ctx_len || p->pool_kernel < 1 || p->curve_points < 2)
+    return LUKV_ERR_INVALID_ARG;
+  if (!(p->softmax_scale >= 0.f) || isinf(p->softmax_scale)) return LUKV_ERR_INVALID_ARG;
+  if (p->head_dim != 64 && p->head_dim != 128) return LUKV_ERR_UNSUPPORTED;
+  if (p->dtype != LUKV_DTYPE_BF16 && p->dtype != LUKV_DTYPE_FP32) return LUKV_ERR_UNSUPPORTED;
+  if ((p->pool_kernel & 1) == 0) return LUKV_ERR_UNSUPPORTED;
+  if (p->curve_points > 4097) return LUKV_ERR_UNSUPPORTED;
+  if (p->ctx_len % (p->curve_points - 1) != 0) return LUKV_ERR_UNSUPPORTED;
+  if ((int64_t)p->gqa_group * p->window > 256) return LUKV_ERR_UNSUPPORTED;
+  const int64_t N = (int64_t)p->n_layers * p->n_kv_heads;
+  const int64_t heads = N * p->batch;
+  // packed row indices, segment ids k*N+hid and grid sizes must fit 32 bits
+  if (heads * p->ctx_len >= (int64_t)1 << 31 || N * (p->curve_points - 1) >= (int64_t)1 << 31 || heads > (1 << 24))
+    return LUKV_ERR_UNSUPPORTED;
+  dm->S = p->batch; dm->L = p->n_layers; dm->H = p->n_kv_heads; dm->G = p->gqa_group; dm->d = p->head_dim;
+  dm->T = p->ctx_len; dm->w = p->window; dm->kp = p->pool_kernel; dm->dtype = p->dtype; dm->P = p->curve_points;
+  dm->N = (int)N;
+  dm->n = dm->T - dm->w;
+  dm->M = dm->G * dm->w;
+  dm->seg = dm->T / (dm->P - 1);
+  dm->nseg = (dm->n + dm->seg - 1) / dm->seg;
+  const float scale = p->softmax_scale > 0.f ? p->softmax_scale : (float)(1.0 / sqrt((double)dm->d));
+  dm->scale_log2 = (float)((double)scale * 1.4426950408889634);
+  return LUKV_OK;
+}
+
+static int check_budgets(const Dims& dm, const int64_t* budgets_in, int64_t* total_rows) {
+  int64_t rows = 0;
+  for (int q = 0; q < dm.S; ++q) {
+    if (budgets_in[q] < 0 || budgets_in[q] > (int64_t)dm.N * dm.n) return LUKV_ERR_BUDGET;
+    rows += budgets_in[q] + (int64_t)dm.N * dm.w;
+  }
+  *total_rows = rows;
+  return LUKV_OK;
+}
+
+static int check_ws(const Dims& dm, void* ws, size_t ws_bytes, Workspace* out) {
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return LUKV_ERR_INVALID_ARG;
+  *out = carve_workspace(dm, ws);
+  if (ws_bytes < out->bytes) return LUKV_ERR_WORKSPACE_TOO_SMALL;
+  return LUKV_OK;
+}
+
+static cudaError_t run_score(const Dims& dm, const void* q, const void* k, const Workspace& ws, float* pooled_out,
+                             LaunchCtx& lc) {
+  cudaError_t e = launch_score_simt(dm, q, k, ws, lc);
+  if (e != cudaSuccess) return e;
+  return launch_pool(dm, ws.raw, pooled_out, lc);
+}
+
+// The whole path on one stream: allocation depends only on the curves, scoring only on Q/K;
+// selection needs both, the gather follows.
+static int run_compress(const Dims& dm, const void* q_win, const void* k, const void* v, const float* curves,
+                        const int64_t* budgets_in, void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets,
+                        int32_t* offsets, int64_t rows_cap, int32_t* dev_status, const Workspace& w, LaunchCtx& lc) {
+  if (dev_status && cudaMemsetAsync(dev_status, 0, sizeof(int32_t), lc.st) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (launch_allocate(dm, curves, budgets_in, w.gains, budgets, offsets, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (run_score(dm, q_win, k, w, w.pooled, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (launch_select(dm, w.pooled, false, budgets, offsets, kept_idx, rows_cap, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (launch_gather(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  return LUKV_OK;
+}
+
+static int check_compress_args(const lukv_params_t* params, const void* q_win, const void* k, const void* v,
+                               const float* curves, const int64_t* budgets_in, void* k_out, void* v_out,
+                               int32_t* kept_idx, int32_t* budgets, int32_t* offsets, int64_t rows_cap, void* ws,
+                               size_t ws_bytes, Dims* dm, Workspace* w) {
+  int rc = make_dims(params, dm);
+  if (rc != LUKV_OK) return rc;
+  if (!q_win || !k || !v || !curves || !budgets_in || !k_out || !v_out || !kept_idx || !budgets || !offsets ||
+      !aligned16(q_win) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
+    return LUKV_ERR_INVALID_ARG;
+  int64_t rows;
+  if ((rc = check_budgets(*dm, budgets_in, &rows)) != LUKV_OK) return rc;
+  if (rows >= (int64_t)1 << 31) return LUKV_ERR_UNSUPPORTED;
+  if (rows_cap < rows) return LUKV_ERR_OUTPUT_TOO_SMALL;
+  return check_ws(*dm, ws, ws_bytes, w);
+}
+
+}  // namespace lukv
+
+using namespace lukv;
+
+extern "C" {
+
+int lukv_workspace_bytes(const lukv_params_t* params, size_t* bytes) {
+  Dims dm;
+  if (!bytes) return LUKV_ERR_INVALID_ARG;
+  const int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  *bytes = carve_workspace(dm, nullptr).bytes;
+  return LUKV_OK;
+}
+
+int lukv_score(const lukv_params_t* params, const void* q_win, const void* k, float* scores, void* ws, size_t ws_bytes,
+               void* stream) {
+  Dims dm;
+  int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (!q_win || !k || !scores || !aligned16(q_win) || !aligned16(k)) return LUKV_ERR_INVALID_ARG;
+  Workspace w;
+  if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  if (run_score(dm, q_win, k, w, scores, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
+}
+
+int lukv_allocate(const lukv_params_t* params, const float* curves, const int64_t* budgets_in, int32_t* budgets,
+                  int32_t* offsets, void* ws, size_t ws_bytes, void* stream) {
+  Dims dm;
+  int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (!curves || !budgets_in || !budgets || !offsets) return LUKV_ERR_INVALID_ARG;
+  int64_t rows;
+  if ((rc = check_budgets(dm, budgets_in, &rows)) != LUKV_OK) return rc;
+  if (rows >= (int64_t)1 << 31) return LUKV_ERR_UNSUPPORTED;
+  Workspace w;
+  if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  if (launch_allocate(dm, curves, budgets_in, w.gains, budgets, offsets, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
+}
+
+int lukv_select_gather(const lukv_params_t* params, const float* scores, const int32_t* budgets, const int32_t* offsets,
+                       const void* k, const void* v, void* k_out, void* v_out, int32_t* kept_idx, int64_t rows_cap,
+                       void* ws, size_t ws_bytes, void* stream) {
+  Dims dm;
+  int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (!scores || !budgets || !offsets || !k || !v || !k_out || !v_out || !kept_idx || rows_cap < 0 || !aligned16(k) ||
+      !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
+    return LUKV_ERR_INVALID_ARG;
+  Workspace w;
+  if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  if (launch_select(dm, scores, false, budgets, offsets, kept_idx, rows_cap, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (launch_gather(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
+}
+
+int lukv_compress(const lukv_params_t* params, const void* q_win, const void* k, const void* v, const float* curves,
+                  const int64_t* budgets_in, void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets,
+                  int32_t* offsets, int64_t rows_cap, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  Dims dm;
+  Workspace w;
+  int rc = check_compress_args(params, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets,
+                               rows_cap, ws, ws_bytes, &dm, &w);
+  if (rc != LUKV_OK) return rc;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  rc = run_compress(dm, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets, rows_cap,
+                    dev_status, w, lc);
+  if (rc == LUKV_OK) g_last_launches = lc.launches;
+  return rc;
+}
+
+int lukv_compress_profile(const lukv_params_t* params, const void* q_win, const void* k, const void* v,
+                          const float* curves, const int64_t* budgets_in, void* k_out, void* v_out,
+                          int32_t* kept_idx, int32_t* budgets, int32_t* offsets, int64_t rows_cap,
+                          int32_t* dev_status, void* ws, size_t ws_bytes, void* stream, lukv_kernel_time_t* times,
+                          int max_times, int* n_times) {
+  Dims dm;
+  Workspace w;
+  if (!times || !n_times || max_times < 1 || max_times > 64) return LUKV_ERR_INVALID_ARG;
+  int rc = check_compress_args(params, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets,
+                               rows_cap, ws, ws_bytes, &dm, &w);
+  if (rc != LUKV_OK) return rc;
+  cudaEvent_t ev[65];
+  const char* names[64];
+  for (int i = 0; i <= max_times; ++i)
+    if (cudaEventCreate(&ev[i]) != cudaSuccess) return LUKV_ERR_CUDA;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  lc.events = ev;
+  lc.names = names;
+  lc.max_events = max_times;
+  cudaEventRecord(ev[0], lc.st);
+  rc = run_compress(dm, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets, rows_cap,
+                    dev_status, w, lc);
+  if (rc == LUKV_OK && cudaStreamSynchronize(lc.st) != cudaSuccess) rc = LUKV_ERR_CUDA;
+  const int cnt = lc.launches < max_times ? lc.launches : max_times;
+  if (rc == LUKV_OK) {
+    for (int i = 0; i < cnt; ++i) {
+      times[i].name = names[i];
+      if (cudaEventElapsedTime(&times[i].ms, ev[i], ev[i + 1]) != cudaSuccess) rc = LUKV_ERR_CUDA;
+    }
+    *n_times = cnt;
+    g_last_launches = lc.launches;
+  }
+  for (int i = 0; i <= max_times; ++i) cudaEventDestroy(ev[i]);
+  return rc;
+}
+
+const char* lukv_strerror(int code) {
+  switch (code) {
+    case LUKV_OK: return "ok";
+    case LUKV_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, non-positive size, flags != 0)";
+    case LUKV_ERR_UNSUPPORTED: return "unsupported configuration (head_dim, dtype, even pool kernel, curve grid, G*w > 256 or sizes beyond 32 bits)";
+    case LUKV_ERR_BUDGET: return "budget outside [0, N*(T-w)]";
+    case LUKV_ERR_WORKSPACE_TOO_SMALL: return "workspace smaller than lukv_workspace_bytes()";
+    case LUKV_ERR_OUTPUT_TOO_SMALL: return "rows_cap smaller than sum(B_q) + S*N*w";
+    case LUKV_ERR_CUDA: return "CUDA launch failed";
+    case LUKV_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+int lukv_last_launch_count(void) { return g_last_launches; }
+
+}  // extern "C"

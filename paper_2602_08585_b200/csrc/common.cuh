@@ -1,0 +1,66 @@
+// Internal declarations shared by the translation units of liblukv.so.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lukv.h"
+
+namespace lukv {
+
+// Problem sizes derived once from lukv_params_t (validated by the API layer).
+struct Dims {
+  int S, L, H, G, d, T, w, kp, dtype, P;
+  int N;        // heads per sequence
+  int n;        // rankable positions per head
+  int M;        // score rows per head = G*w
+  int seg;      // tokens per curve segment s = T/(P-1)
+  int nseg;     // curve segments with non-zero capacity = ceil(n/seg)
+  float scale_log2;  // softmax scale * log2(e): logits are kept in the exp2 domain
+  int64_t heads() const { return (int64_t)S * N; }
+  size_t esize() const { return dtype == LUKV_DTYPE_BF16 ? 2 : 4; }
+};
+
+// Workspace carve-up (all offsets 256-byte aligned).
+struct Workspace {
+  float* raw;        // [S*N][n]   un-pooled scores
+  float* pooled;     // [S*N][n]   pooled scores (fused path)
+  float* stats;      // [S*N][chunks][M][2] partial (max, sum) of the SIMT scorer
+  float* lse;        // [S*N][M]   row log-sum-exp in the exp2 domain
+  float* gains;      // [N][P-1]   hull gains
+  size_t bytes;
+};
+
+int score_chunks(const Dims& dm);                       // key chunks per head of the SIMT scorer
+Workspace carve_workspace(const Dims& dm, void* base);  // base may be null (size query)
+
+// Launch bookkeeping: counts the kernels a call enqueues and, when a timeline is attached
+// (profiling entry point only), records a CUDA event after each of them.
+struct LaunchCtx {
+  cudaStream_t st = nullptr;
+  int launches = 0;
+  cudaEvent_t* events = nullptr;  // [max_events + 1]; events[0] is recorded by the caller
+  const char** names = nullptr;   // [max_events]
+  int max_events = 0;
+  void mark(const char* name) {
+    if (events && launches < max_events) {
+      names[launches] = name;
+      cudaEventRecord(events[launches + 1], st);
+    }
+    ++launches;
+  }
+};
+
+// Launchers.  Each returns cudaGetLastError() after its launches.
+cudaError_t launch_score_simt(const Dims& dm, const void* q, const void* k, const Workspace& ws, LaunchCtx& lc);
+cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, LaunchCtx& lc);
+cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, float* gains,
+                            int32_t* budgets, int32_t* offsets, LaunchCtx& lc);
+// scores_are_raw: apply the max-pool while loading (fused path) instead of expecting pooled input
+cudaError_t launch_select(const Dims& dm, const float* scores, bool scores_are_raw, const int32_t* budgets,
+                          const int32_t* offsets, int32_t* kept_idx, int64_t rows_cap, LaunchCtx& lc);
+cudaError_t launch_gather(const Dims& dm, const int32_t* offsets, const int32_t* kept_idx, const void* k,
+                          const void* v, void* k_out, void* v_out, int64_t rows_cap, LaunchCtx& lc);
+
+}  // namespace lukv

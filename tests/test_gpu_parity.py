@@ -1,0 +1,239 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Bars: scores within max relative error 2e-3 (+1e-30 absolute at the underflow edge);
+allocation, selection and gather bit-exact when run on the oracle's own curves and scores;
+end-to-end kept-index agreement >= 99.9 % with every mismatch at a score gap below the
+tolerance.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_08585_b200 import lukv, synth
+from gpu_helpers import (assert_scores_close, bits, gpu_allocate, gpu_compress, gpu_score, gpu_select_gather,
+                         kept_agreement, params_of)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    lukv.lib()
+
+
+def _rand_qkv(S, L, H, G, d, T, w, dtype, seed, scale=1.0):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    q = (torch.randn((S, L, H * G, w, d), generator=g) * scale).to(dtype)
+    k = (torch.randn((S, L, H, T, d), generator=g) * scale).to(dtype)
+    v = torch.randn((S, L, H, T, d), generator=g).to(dtype)
+    return q, k, v
+
+
+# ---- stage (a): scores -------------------------------------------------------------------------
+
+SCORE_SHAPES = [
+    # S, L, H, G, d,   T,   w, kp, dtype
+    (1, 1, 1, 1, 64, 2, 1, 1, torch.float32),          # smallest legal problem
+    (1, 1, 2, 1, 64, 77, 5, 3, torch.float32),         # ragged everything
+    (2, 1, 2, 3, 64, 1025, 7, 5, torch.bfloat16),      # one key past a chunk
+    (1, 2, 1, 4, 128, 1300, 32, 7, torch.bfloat16),    # 128 rows, ragged tail
+    (1, 1, 1, 7, 128, 2048, 32, 7, torch.bfloat16),    # 224 rows (GQA group 7)
+    (1, 1, 1, 4, 128, 1111, 64, 5, torch.bfloat16),    # 256 rows
+    (1, 1, 2, 2, 128, 640, 16, 9, torch.float32),
+    (1, 1, 1, 1, 128, 4096 + 33, 33, 1, torch.bfloat16),
+]
+
+
+@pytest.mark.parametrize("shape", SCORE_SHAPES)
+def test_score_matches_oracle(oracle, shape):
+    S, L, H, G, d, T, w, kp, dtype = shape
+    q, k, _ = _rand_qkv(S, L, H, G, d, T, w, dtype, seed=T + w, scale=2.0)
+    p = lukv.make_params(S, L, H, G, d, T, w, kp, dtype, 2)
+    got = gpu_score(p, q.cuda(), k.cuda()).cpu().numpy()
+    ref = oracle.score(bits(q), bits(k), G, kp)
+    assert_scores_close(got, ref)
+
+
+def test_score_explicit_scale(oracle):
+    S, L, H, G, d, T, w, kp = 1, 1, 2, 2, 64, 300, 4, 3
+    q, k, _ = _rand_qkv(S, L, H, G, d, T, w, torch.bfloat16, seed=5)
+    p = lukv.make_params(S, L, H, G, d, T, w, kp, torch.bfloat16, 2, scale=0.3)
+    got = gpu_score(p, q.cuda(), k.cuda()).cpu().numpy()
+    assert_scores_close(got, oracle.score(bits(q), bits(k), G, kp, scale=0.3))
+
+
+@pytest.mark.parametrize("name", ["tiny", "llama8b_1layer_8k"])
+def test_score_on_benchmark_configs(oracle, name):
+    wl = synth.CONFIGS[name]
+    q, k, _ = synth.gen_tensors(wl, "cuda")
+    qc, kc, _ = synth.gen_tensors(wl, "cpu")
+    assert torch.equal(q.cpu(), qc) and torch.equal(k.cpu(), kc)      # same bits on both devices
+    got = gpu_score(params_of(wl), q, k).cpu().numpy()
+    ref = oracle.score(bits(qc), bits(kc), wl.G, wl.kp)
+    assert_scores_close(got, ref)
+
+
+# ---- stage (b): allocation ---------------------------------------------------------------------
+
+def _alloc_case(oracle, N, P, T, w, curves, Bs, L=None):
+    L = L or 1
+    p = lukv.make_params(len(Bs), L, N // L, 1, 64, T, w, 1, torch.bfloat16, P)
+    b_gpu, o_gpu = gpu_allocate(p, curves, Bs)
+    b_ref, o_ref = oracle.allocate(curves, T, w, Bs)
+    np.testing.assert_array_equal(b_gpu, b_ref)
+    np.testing.assert_array_equal(o_gpu, o_ref)
+
+
+@pytest.mark.parametrize("name", list(synth.CONFIGS))
+def test_allocate_bit_exact_on_benchmark_configs(oracle, name):
+    wl = synth.CONFIGS[name]
+    curves = synth.gen_curves(wl)
+    p = params_of(wl)
+    b_gpu, o_gpu = gpu_allocate(p, curves, wl.budgets())
+    b_ref, o_ref = oracle.allocate(curves, wl.T, wl.w, wl.budgets())
+    np.testing.assert_array_equal(b_gpu, b_ref)
+    np.testing.assert_array_equal(o_gpu, o_ref)
+    np.testing.assert_array_equal(b_gpu.sum(axis=1), wl.budgets())
+    assert o_gpu[-1] == wl.total_rows()
+
+
+def test_allocate_edge_cases(oracle):
+    rng = np.random.default_rng(0)
+    N, P, T, w = 12, 9, 64, 5          # s = 8, n = 59: last segment holds 3 tokens
+    inc = rng.exponential(size=(N, P - 1))
+    U = np.zeros((N, P), np.float32)
+    U[:, 1:] = np.cumsum(inc, axis=1)
+    n = T - w
+    _alloc_case(oracle, N, P, T, w, U, [0, 1, 100, 333, N * n - 1, N * n])
+    # flat and identical curves: every gain ties, order falls back to (k, hid)
+    flat = np.tile(np.arange(P, dtype=np.float32), (N, 1))
+    _alloc_case(oracle, N, P, T, w, flat, [7, 8 * N + 3, 50 * N + 1, N * n])
+    # concave, integer valued (exact ties between heads), decreasing tails (zero gains)
+    conc = np.zeros((N, P), np.float32)
+    conc[:, 1:] = np.cumsum(np.arange(P - 1, 0, -1, dtype=np.float64))[None, :]
+    _alloc_case(oracle, N, P, T, w, conc, [N * 8 * 3, 100, 401])
+    dip = U.copy()
+    dip[:, 5:] -= np.arange(1, P - 4, dtype=np.float32)[None, :] * 3.0
+    _alloc_case(oracle, N, P, T, w, dip, [50, 300, N * n])
+    # window wider than a segment: several trailing segments are unusable
+    _alloc_case(oracle, N, 17, 64, 21, np.ascontiguousarray(np.repeat(U, 2, axis=1)[:, :17]), [10, 200, N * 43])
+    # all-zero curves (every gain is +0)
+    _alloc_case(oracle, N, P, T, w, np.zeros((N, P), np.float32), [0, 77, N * n])
+
+
+def test_allocate_many_sequences_and_many_heads(oracle):
+    rng = np.random.default_rng(1)
+    N, P, T, w = 300, 33, 1024, 16     # more heads than threads of one allocation CTA
+    inc = rng.exponential(size=(N, P - 1)) * np.where(rng.random((N, P - 1)) < 0.2, 3.0, 1.0)
+    U = np.zeros((N, P), np.float32)
+    U[:, 1:] = np.cumsum(inc, axis=1)
+    Bs = [int(x) for x in rng.integers(0, N * (T - w), size=40)]     # more sequences than one launch takes
+    _alloc_case(oracle, N, P, T, w, U, Bs, L=3)
+
+
+def test_allocate_long_curves(oracle):
+    rng = np.random.default_rng(2)
+    N, P, T, w = 5, 4097, 4096, 32
+    inc = rng.exponential(size=(N, P - 1)) * np.where(rng.random((N, P - 1)) < 0.2, 3.0, 1.0)
+    U = np.zeros((N, P), np.float32)
+    U[:, 1:] = np.cumsum(inc, axis=1)
+    _alloc_case(oracle, N, P, T, w, U, [1234, 9999])
+
+
+# ---- stages (c)+(d): selection and gather on the oracle's scores ------------------------------------
+
+def _select_case(oracle, S, N, T, w, d, dtype, budgets, scores, seed=0):
+    g = torch.Generator().manual_seed(seed)
+    k = torch.randn((S, 1, N, T, d), generator=g).to(dtype)
+    v = torch.randn((S, 1, N, T, d), generator=g).to(dtype)
+    budgets = np.asarray(budgets, np.int32).reshape(S, N)
+    offsets = np.concatenate([[0], np.cumsum(budgets.reshape(-1) + w)]).astype(np.int32)
+    rows = int(offsets[-1])
+    p = lukv.make_params(S, 1, N, 1, d, T, w, 1, dtype, 2)
+    k_out, v_out, kept = gpu_select_gather(p, torch.from_numpy(scores).cuda(), torch.from_numpy(budgets).cuda(),
+                                           torch.from_numpy(offsets).cuda(), k.cuda(), v.cuda(), rows, pad_rows=3)
+    rk, rv, rkept = oracle.select_gather(scores.reshape(S * N, T - w), budgets, offsets, bits(k).reshape(S * N, T, d),
+                                         bits(v).reshape(S * N, T, d), w)
+    np.testing.assert_array_equal(kept.cpu().numpy()[:rows], rkept)
+    np.testing.assert_array_equal(bits(k_out)[:rows], rk)
+    np.testing.assert_array_equal(bits(v_out)[:rows], rv)
+    # rows beyond rows_cap are never written
+    assert torch.all(kept[rows:] == -1) and torch.all(k_out[rows:] == 0) and torch.all(v_out[rows:] == 0)
+
+
+@pytest.mark.parametrize("T,w,d,dtype", [(77, 5, 64, torch.float32), (1024, 16, 64, torch.float32),
+                                         (5000, 32, 128, torch.bfloat16), (20000, 32, 128, torch.bfloat16),
+                                         (33000, 64, 64, torch.bfloat16), (40000, 32, 128, torch.float32)])
+def test_select_gather_bit_exact(oracle, T, w, d, dtype):
+    rng = np.random.default_rng(T)
+    S, N, n = 2, 3, T - w
+    scores = rng.random((S, N, n)).astype(np.float32) ** 8
+    scores[0, 1] = np.repeat(rng.random(n // 7 + 1).astype(np.float32), 7)[:n]     # plateaus: ties at the cut
+    scores[1, 0] = 0.0                                                               # all equal
+    scores[1, 2, ::3] = 0.0
+    budgets = [0, n // 3, n, 17 % n, 1, n - 1]
+    _select_case(oracle, S, N, T, w, d, dtype, budgets, scores, seed=T)
+
+
+def test_select_gather_long_context_single_head(oracle):
+    T, w, d = 131072, 32, 128
+    rng = np.random.default_rng(9)
+    scores = np.maximum(rng.standard_normal((1, 1, T - w)).astype(np.float32), 0.0)   # half the scores tie at 0
+    _select_case(oracle, 1, 1, T, w, d, torch.bfloat16, [90000], scores)
+
+
+# ---- the whole path ------------------------------------------------------------------------------
+
+def _compress_case(oracle, wl, min_agreement=0.999):
+    q, k, v = synth.gen_tensors(wl, "cuda")
+    curves = synth.gen_curves(wl)
+    Bs = wl.budgets()
+    out = gpu_compress(params_of(wl), q, k, v, curves, Bs)
+    ref = oracle.compress(bits(q), bits(k), bits(v), curves, Bs, wl.G, wl.kp)
+    budgets = out.budgets.cpu().numpy()
+    offsets = out.offsets.cpu().numpy()
+    kept = out.kept_idx.cpu().numpy()
+    np.testing.assert_array_equal(budgets, ref["budgets"])
+    np.testing.assert_array_equal(offsets, ref["offsets"])
+    agree = kept_agreement(kept, ref["kept_idx"], offsets, budgets, ref["scores"])
+    assert agree >= min_agreement, f"kept-index agreement {agree:.5f}"
+    # packed rows are bit-exact copies of the rows kept_idx names (window rows included)
+    kb, vb = bits(k).reshape(wl.S * wl.N, wl.T, wl.d), bits(v).reshape(wl.S * wl.N, wl.T, wl.d)
+    ko, vo = bits(out.k_out), bits(out.v_out)
+    for u in range(wl.S * wl.N):
+        lo, hi = offsets[u], offsets[u + 1]
+        np.testing.assert_array_equal(ko[lo:hi], kb[u][kept[lo:hi]])
+        np.testing.assert_array_equal(vo[lo:hi], vb[u][kept[lo:hi]])
+        np.testing.assert_array_equal(kept[hi - wl.w:hi], np.arange(wl.n, wl.T))
+    # identical index sets => identical packed bytes
+    same = kept == ref["kept_idx"]
+    np.testing.assert_array_equal(ko[same], ref["k_out"][same])
+    np.testing.assert_array_equal(vo[same], ref["v_out"][same])
+    return agree
+
+
+@pytest.mark.parametrize("name", ["tiny", "llama8b_1layer_8k"])
+def test_compress_on_benchmark_configs(oracle, name):
+    _compress_case(oracle, synth.CONFIGS[name])
+
+
+def test_compress_reduced_batch_mixed_budgets(oracle):
+    # the batched mixed-budget configuration at reduced size: 2 layers x 2 heads, 4 sequences
+    wl = synth.scaled(synth.CONFIGS["batch8_16k_mixed"], S=4, L=2, H=2, T=2048, P=33, needles=16)
+    _compress_case(oracle, wl)
+
+
+def test_compress_reduced_gqa7_student_t(oracle):
+    wl = synth.scaled(synth.CONFIGS["gqa7_128k"], L=1, H=2, T=4096, P=65, needles=32)
+    _compress_case(oracle, wl)
+
+
+def test_compress_is_deterministic():
+    wl = synth.scaled(synth.CONFIGS["llama8b_1layer_8k"], H=2, T=4096, P=65)
+    q, k, v = synth.gen_tensors(wl, "cuda")
+    curves = synth.gen_curves(wl)
+    a = gpu_compress(params_of(wl), q, k, v, curves, wl.budgets())
+    b = gpu_compress(params_of(wl), q, k, v, curves, wl.budgets())
+    assert torch.equal(a.kept_idx, b.kept_idx) and torch.equal(a.k_out.view(torch.int16), b.k_out.view(torch.int16))
+    assert torch.equal(a.budgets, b.budgets) and torch.equal(a.offsets, b.offsets)
