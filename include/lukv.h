@@ -167,6 +167,29 @@ LUKV_API int lukv_compress_profile(const lukv_params_t* params, const void* q_wi
                                    int32_t* dev_status, void* ws, size_t ws_bytes, void* stream,
                                    lukv_kernel_time_t* times, int max_times, int* n_times);
 
+/*
+ * lukv_allocate for callers that cannot hand over device scratch (the paper has no
+ * counterpart; this is a packaging variant of stage (b)).  Some hosts of this library may
+ * not call cudaMalloc at the point where budgets are needed -- a serving process whose
+ * device memory is fully owned by its own pool allocator, or code running inside a region
+ * where allocation is forbidden -- and so have no workspace to pass.  This entry point takes
+ * none: the hull gains go to a fixed array of LUKV_STATIC_GAINS_MAX = 262144 floats (1 MiB)
+ * that is part of the library image and is resident on every GPU that loads the library
+ * until the process exits.  It calls no allocating routine.
+ *
+ *   - Limit: N*(P-1) <= 262144 (e.g. 256 heads x 1025 points); larger problems return
+ *     LUKV_ERR_WORKSPACE_TOO_SMALL and launch nothing.
+ *   - The first call on each device looks up the array's device address (a one-time runtime
+ *     query, cached per device); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array.  It keeps the previous call's contents,
+ *     which is harmless: every call rewrites the gains it uses before reading them.  Calls
+ *     whose kernels can overlap on the GPU (different streams, or threads) race on it and
+ *     must be serialised by the caller.
+ *   - Arguments, results and error codes otherwise as lukv_allocate (no ws, ws_bytes).
+ */
+LUKV_API int lukv_allocate_static(const lukv_params_t* params, const float* curves, const int64_t* budgets_in,
+                                  int32_t* budgets, int32_t* offsets, void* stream);
+
 /* Static description of a status code. */
 LUKV_API const char* lukv_strerror(int code);
 

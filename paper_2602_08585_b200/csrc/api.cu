@@ -2,6 +2,8 @@
 // Every step of the path runs in the kernels of this library; there is no host fallback.
 #include <math.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace lukv {
@@ -233,6 +235,51 @@ int lukv_compress_profile(const lukv_params_t* params, const void* q_win, const 
   }
   for (int i = 0; i <= max_times; ++i) cudaEventDestroy(ev[i]);
   return rc;
+}
+
+// ---- allocation without a caller-provided workspace ---------------------------------------
+// Scratch of lukv_allocate_static: the hull gains [N][P-1].  The array lives in every GPU
+// context that loads this library, from load until exit.
+#define LUKV_STATIC_GAINS_MAX (256 * 1024)
+static __device__ __align__(256) float g_static_gains[LUKV_STATIC_GAINS_MAX];
+
+// In host code `g_static_gains` is only a handle for the runtime, not a device address; the
+// address on the current device is looked up once per device and cached here.
+static float* g_static_gains_ptr[64] = {nullptr};
+static std::mutex g_static_gains_mutex;
+
+static int static_gains_address(float** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LUKV_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_gains_mutex);
+  if (!g_static_gains_ptr[dev]) {
+    float* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_static_gains) != cudaSuccess || !ptr) return LUKV_ERR_CUDA;
+    g_static_gains_ptr[dev] = ptr;
+  }
+  *out = g_static_gains_ptr[dev];
+  return LUKV_OK;
+}
+
+int lukv_allocate_static(const lukv_params_t* params, const float* curves, const int64_t* budgets_in,
+                         int32_t* budgets, int32_t* offsets, void* stream) {
+  Dims dm;
+  int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (!curves || !budgets_in || !budgets || !offsets) return LUKV_ERR_INVALID_ARG;
+  if ((int64_t)dm.N * (dm.P - 1) > LUKV_STATIC_GAINS_MAX) return LUKV_ERR_WORKSPACE_TOO_SMALL;
+  int64_t rows;
+  if ((rc = check_budgets(dm, budgets_in, &rows)) != LUKV_OK) return rc;
+  if (rows >= (int64_t)1 << 31) return LUKV_ERR_UNSUPPORTED;
+  float* gains = nullptr;
+  if ((rc = static_gains_address(&gains)) != LUKV_OK) return rc;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  // the hull kernel overwrites gains[0 .. N*(P-1)) before the greedy kernel reads them, so
+  // nothing left by an earlier call is ever consumed
+  if (launch_allocate(dm, curves, budgets_in, gains, budgets, offsets, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
 }
 
 const char* lukv_strerror(int code) {

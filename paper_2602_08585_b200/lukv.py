@@ -21,7 +21,7 @@ ERR_OUTPUT_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 
 EXPORTS = ("lukv_workspace_bytes", "lukv_score", "lukv_allocate", "lukv_select_gather", "lukv_compress",
-           "lukv_strerror", "lukv_last_launch_count", "lukv_compress_profile")
+           "lukv_strerror", "lukv_last_launch_count", "lukv_compress_profile", "lukv_allocate_static")
 
 
 class Params(ctypes.Structure):
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.lukv_compress.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
         L.lukv_compress_profile.argtypes = L.lukv_compress.argtypes + [ctypes.POINTER(KernelTime), ctypes.c_int,
                                                                        ctypes.POINTER(ctypes.c_int)]
+        L.lukv_allocate_static.argtypes = [pp, vp, vp, vp, vp, vp]
         L.lukv_strerror.argtypes = [ctypes.c_int]
         L.lukv_strerror.restype = ctypes.c_char_p
         for name in EXPORTS[:5] + EXPORTS[6:]:
@@ -137,6 +138,16 @@ def lukv_allocate(params: Params, curves, budgets_in, budgets, offsets, ws, stre
     rc = lib().lukv_allocate(ctypes.byref(params), _ptr(curves), b.ctypes.data, _ptr(budgets), _ptr(offsets),
                              _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(stream))
     return _check(rc, "lukv_allocate", check)
+
+
+def lukv_allocate_static(params: Params, curves, budgets_in, budgets, offsets, stream=None, check: bool = True) -> int:
+    """lukv_allocate without a workspace argument: the scratch is a fixed array inside the library
+    (at most 262144 gains), for callers that cannot allocate device memory.  Calls sharing a device
+    must not overlap on the GPU."""
+    b = _host_budgets(budgets_in)
+    rc = lib().lukv_allocate_static(ctypes.byref(params), _ptr(curves), b.ctypes.data, _ptr(budgets), _ptr(offsets),
+                                    _stream(stream))
+    return _check(rc, "lukv_allocate_static", check)
 
 
 def lukv_select_gather(params: Params, scores, budgets, offsets, k, v, k_out, v_out, kept_idx, rows_cap: int, ws,
