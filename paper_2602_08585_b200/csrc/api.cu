@@ -1,6 +1,7 @@
 // C ABI of liblukv.so: argument validation, workspace carve-up and stage sequencing.
 // Every step of the path runs in the kernels of this library; there is no host fallback.
 #include <math.h>
+#include <stdlib.h>
 
 #include <mutex>
 
@@ -81,9 +82,19 @@ static int check_ws(const Dims& dm, void* ws, size_t ws_bytes, Workspace* out) {
   return LUKV_OK;
 }
 
+// LUKV_FORCE_SIMT=1 routes every shape through the FP32-pipe scorer (for A/B checks).
+static bool force_simt() {
+  static const bool v = [] {
+    const char* e = getenv("LUKV_FORCE_SIMT");
+    return e && e[0] == '1';
+  }();
+  return v;
+}
+
 static cudaError_t run_score(const Dims& dm, const void* q, const void* k, const Workspace& ws, float* pooled_out,
-                             LaunchCtx& lc) {
-  cudaError_t e = launch_score_simt(dm, q, k, ws, lc);
+                             int32_t* dev_status, LaunchCtx& lc) {
+  cudaError_t e = (score_tc_supported(dm) && !force_simt()) ? launch_score_tc(dm, q, k, ws, dev_status, lc)
+                                                            : launch_score_simt(dm, q, k, ws, lc);
   if (e != cudaSuccess) return e;
   return launch_pool(dm, ws.raw, pooled_out, lc);
 }
@@ -95,7 +106,7 @@ static int run_compress(const Dims& dm, const void* q_win, const void* k, const 
                         int32_t* offsets, int64_t rows_cap, int32_t* dev_status, const Workspace& w, LaunchCtx& lc) {
   if (dev_status && cudaMemsetAsync(dev_status, 0, sizeof(int32_t), lc.st) != cudaSuccess) return LUKV_ERR_CUDA;
   if (launch_allocate(dm, curves, budgets_in, w.gains, budgets, offsets, lc) != cudaSuccess) return LUKV_ERR_CUDA;
-  if (run_score(dm, q_win, k, w, w.pooled, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (run_score(dm, q_win, k, w, w.pooled, dev_status, lc) != cudaSuccess) return LUKV_ERR_CUDA;
   if (launch_select(dm, w.pooled, false, budgets, offsets, kept_idx, rows_cap, lc) != cudaSuccess) return LUKV_ERR_CUDA;
   if (launch_gather(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, lc) != cudaSuccess) return LUKV_ERR_CUDA;
   return LUKV_OK;
@@ -142,7 +153,7 @@ int lukv_score(const lukv_params_t* params, const void* q_win, const void* k, fl
   if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;
-  if (run_score(dm, q_win, k, w, scores, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (run_score(dm, q_win, k, w, scores, nullptr, lc) != cudaSuccess) return LUKV_ERR_CUDA;
   g_last_launches = lc.launches;
   return LUKV_OK;
 }

@@ -54,6 +54,12 @@ struct LaunchCtx {
 
 // Launchers.  Each returns cudaGetLastError() after its launches.
 cudaError_t launch_score_simt(const Dims& dm, const void* q, const void* k, const Workspace& ws, LaunchCtx& lc);
+// Folds per-chunk (max, sum-exp) partials [heads][chunks][M][2] into lse[heads][M] (exp2 domain).
+cudaError_t launch_lse(const Dims& dm, const float* stats, float* lse, int chunks, LaunchCtx& lc);
+// Tensor-core scorer (bf16, head_dim 128).  dev_status may be null.
+bool score_tc_supported(const Dims& dm);
+cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const Workspace& ws, int32_t* dev_status,
+                            LaunchCtx& lc);
 cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, LaunchCtx& lc);
 cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, float* gains,
                             int32_t* budgets, int32_t* offsets, LaunchCtx& lc);

@@ -254,6 +254,12 @@ cudaError_t launch_score_simt(const Dims& dm, const void* q, const void* k, cons
   return dispatch_rows<float, 128>(dm, q, k, ws, lc);
 }
 
+cudaError_t launch_lse(const Dims& dm, const float* stats, float* lse, int chunks, LaunchCtx& lc) {
+  score_lse_kernel<<<(unsigned)dm.heads(), 256, 0, lc.st>>>(stats, lse, dm.M, chunks);
+  lc.mark("score_lse");
+  return cudaGetLastError();
+}
+
 cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, LaunchCtx& lc) {
   const int tiles = (dm.n + 255) / 256;
   max_pool_kernel<<<(unsigned)(dm.heads() * tiles), 256, 0, lc.st>>>(raw, pooled, dm.n, dm.kp / 2, tiles);
