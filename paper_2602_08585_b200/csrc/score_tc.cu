@@ -131,8 +131,9 @@ struct SmemPlan {
   static constexpr int kBarOff = kQBytes + kStages * kStageBytes;
   // barriers: full[kStages], empty[kStages], tfull[2], tempty[2], qfull
   static constexpr int kNumBars = 2 * kStages + 5;
-  static constexpr int kMiscOff = kBarOff + kNumBars * 8;  // tmem base (4 B), abort flag (4 B)
-  static constexpr int kLseOff = kMiscOff + 16;            // sweep 2: lse of up to 256 rows
+  static constexpr int kMiscOff = (kBarOff + kNumBars * 8 + 15) & ~15;  // tmem base (4 B), abort flag (4 B)
+  static constexpr int kLseOff = kMiscOff + 16;            // sweep 2: lse of up to 256 rows (read as float4: 16-byte aligned)
+  static_assert(kLseOff % 16 == 0, "lse rows are read with 16-byte loads");
   static constexpr int kPartOff = kLseOff + 256 * 4;       // sweep 1, MT==1: (m,l) of the second quad
   static constexpr int kTotal = kPartOff + 128 * 8 + 1024;  // + slack for the 1024-byte alignment
 };
