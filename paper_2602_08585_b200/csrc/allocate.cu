@@ -26,60 +26,63 @@ __device__ __forceinline__ bool mean_le(double a, double b, double c, double d) 
   return __ddiv_rn(a, b) <= __ddiv_rn(c, d);
 }
 
-// One thread per head; a block stages `hb` heads in shared memory, interleaved by head so
-// that every thread stays in its own bank.  Stack entries are block start points; a
-// block's end is the next entry's start.
-__global__ void hull_kernel(const float* __restrict__ curves, float* __restrict__ gains, int N, int P, int hb) {
+// One warp per head.  Lane 0 runs the pool-adjacent-violators stack (the sequence of merge
+// decisions is the algorithm; it is serial by nature) with the top block cached in registers;
+// the other lanes stage the curve into shared memory and write the gains out.
+// Stack entries are block start points; a block's end is the next entry's start.
+__global__ void hull_kernel(const float* __restrict__ curves, float* __restrict__ gains, int N, int P) {
   extern __shared__ __align__(16) unsigned char hull_smem[];
-  float* Us = reinterpret_cast<float*>(hull_smem);   // [P][hb]; overwritten by the gains
-  int* Ls = reinterpret_cast<int*>(Us + (size_t)P * hb);  // [P][hb]
-  const int hid0 = blockIdx.x * hb;
-  const int heads_here = min(hb, N - hid0);
-  for (int i = threadIdx.x; i < heads_here * P; i += blockDim.x) {
-    const int h = i / P, p = i % P;
-    Us[p * hb + h] = curves[(size_t)(hid0 + h) * P + p];
-  }
-  __syncthreads();
-  const int h = threadIdx.x;
-  if (h < heads_here) {
-    int sp = 0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warps = blockDim.x >> 5;
+  const int hid = blockIdx.x * warps + warp;
+  if (hid >= N) return;  // whole warps leave together; only __syncwarp is used below
+  float* Us = reinterpret_cast<float*>(hull_smem) + (size_t)warp * 3 * P;  // [P] curve
+  int* Ls = reinterpret_cast<int*>(Us + P);                                // [P] stack of block starts
+  float* Gs = Us + 2 * P;                                                   // [P-1] gains
+  for (int p = lane; p < P; p += 32) Us[p] = curves[(size_t)hid * P + p];
+  __syncwarp();
+  int sp = 0;
+  if (lane == 0) {
+    int top_l = 0;
+    double top_num = 0.0, top_den = 1.0;
     for (int k = 0; k + 1 < P; ++k) {
       int cur_l = k;
-      const int cur_r = k + 1;
-      const double u_r = (double)Us[cur_r * hb + h];
-      double cur_num = __dsub_rn(u_r, (double)Us[cur_l * hb + h]);
+      const double u_r = (double)Us[k + 1];
+      double cur_num = __dsub_rn(u_r, (double)Us[k]);
       double cur_den = 1.0;
-      while (sp > 0) {
-        const int top_l = Ls[(sp - 1) * hb + h];
-        const double top_num = __dsub_rn((double)Us[cur_l * hb + h], (double)Us[top_l * hb + h]);
-        const double top_den = (double)(cur_l - top_l);
-        if (!mean_le(top_num, top_den, cur_num, cur_den)) break;
+      while (sp > 0 && mean_le(top_num, top_den, cur_num, cur_den)) {
         cur_l = top_l;
         --sp;
-        cur_num = __dsub_rn(u_r, (double)Us[cur_l * hb + h]);
-        cur_den = (double)(cur_r - cur_l);
+        cur_num = __dsub_rn(u_r, (double)Us[cur_l]);
+        cur_den = (double)(k + 1 - cur_l);
+        if (sp > 0) {
+          top_l = Ls[sp - 1];
+          top_num = __dsub_rn((double)Us[cur_l], (double)Us[top_l]);
+          top_den = (double)(cur_l - top_l);
+        }
       }
-      Ls[sp * hb + h] = cur_l;
-      ++sp;
-    }
-    for (int i = 0; i < sp; ++i) {
-      const int l = Ls[i * hb + h];
-      const int r = (i + 1 < sp) ? Ls[(i + 1) * hb + h] : P - 1;
-      const double mean = __ddiv_rn(__dsub_rn((double)Us[r * hb + h], (double)Us[l * hb + h]), (double)(r - l));
-      const float g = __double2float_rn(mean > 0.0 ? mean : 0.0);
-      for (int k = l; k < r; ++k) Us[k * hb + h] = g;  // U[l..r-1] are no longer needed
+      Ls[sp++] = cur_l;
+      top_l = cur_l;
+      top_num = cur_num;
+      top_den = cur_den;
     }
   }
-  __syncthreads();
-  for (int i = threadIdx.x; i < heads_here * (P - 1); i += blockDim.x) {
-    const int hh = i / (P - 1), kk = i % (P - 1);
-    gains[(size_t)(hid0 + hh) * (P - 1) + kk] = Us[kk * hb + hh];
+  sp = __shfl_sync(0xffffffffu, sp, 0);
+  __syncwarp();
+  for (int i = lane; i < sp; i += 32) {
+    const int l = Ls[i];
+    const int r = (i + 1 < sp) ? Ls[i + 1] : P - 1;
+    const double mean = __ddiv_rn(__dsub_rn((double)Us[r], (double)Us[l]), (double)(r - l));
+    const float g = __double2float_rn(mean > 0.0 ? mean : 0.0);
+    for (int k = l; k < r; ++k) Gs[k] = g;
   }
+  __syncwarp();
+  for (int k = lane; k + 1 < P; k += 32) gains[(size_t)hid * (P - 1) + k] = Gs[k];
 }
 
 // ---- greedy --------------------------------------------------------------------------
 
-constexpr int kGreedyThreads = 256;
+constexpr int kGreedyThreads = 1024;
 constexpr int kSeqPerLaunch = 32;
 
 struct GreedyArgs {
@@ -103,14 +106,16 @@ __device__ __forceinline__ long long capsum(int c, int seg, int n) {  // tokens 
 // before lo are already bought.  Each of the 8 passes histograms the next key byte of the
 // active segments weighted by capacity, picks the byte at which the remaining budget runs
 // out and narrows every head's range to it.  Keys are unique, so one segment remains: the
-// partially bought one.
+// partially bought one.  `tph` threads (a power of two) share a head and split its range.
 __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __restrict__ gains, GreedyArgs args,
                                                                 int32_t* __restrict__ budgets,
                                                                 int32_t* __restrict__ offsets, int N, int P, int seg,
-                                                                int nseg, int n, int w) {
+                                                                int nseg, int n, int w, int tph) {
   extern __shared__ __align__(16) unsigned char greedy_smem[];
   int* lo = reinterpret_cast<int*>(greedy_smem);  // [N]
   int* hi = lo + N;                               // [N]
+  int* cnt_lt = hi + N;                           // [N] active segments with byte <  chosen byte
+  int* cnt_le = cnt_lt + N;                       // [N] active segments with byte <= chosen byte
   __shared__ unsigned long long hist[256];
   __shared__ long long sh_remaining;
   __shared__ int sh_digit, sh_all_taken;
@@ -119,6 +124,8 @@ __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __r
   const int q = args.seq0 + blockIdx.x;
   const int tid = threadIdx.x;
   const int G1 = P - 1;
+  const int sub = tid & (tph - 1);           // this thread's share of a head
+  const int heads_per_iter = kGreedyThreads / tph;
   for (int h = tid; h < N; h += kGreedyThreads) {
     lo[h] = 0;
     hi[h] = nseg;
@@ -131,23 +138,39 @@ __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __r
 
   for (int pass = 0; pass < 8; ++pass) {
     const int shift = 56 - 8 * pass;
-    hist[tid] = 0ull;  // kGreedyThreads == 256 bins
-    __syncthreads();
+    if (tid < 256) hist[tid] = 0ull;
     for (int h = tid; h < N; h += kGreedyThreads) {
+      cnt_lt[h] = 0;
+      cnt_le[h] = 0;
+    }
+    __syncthreads();
+    for (int h = tid / tph; h < N; h += heads_per_iter) {
       const int l = lo[h], r = hi[h];
-      if (l >= r) continue;
+      const int len = r - l;
+      const int a = l + (int)(((long long)len * sub) / tph), b = l + (int)(((long long)len * (sub + 1)) / tph);
+      if (a >= b) continue;
       const float* g = gains + (size_t)h * G1;
-      int run_start = l;
-      unsigned run_digit = (unsigned)(seg_key(__ldg(g + l), l, h, N) >> shift) & 255u;
-      for (int k = l + 1; k < r; ++k) {
-        const unsigned dgt = (unsigned)(seg_key(__ldg(g + k), k, h, N) >> shift) & 255u;
-        if (dgt != run_digit) {
-          atomicAdd(&hist[run_digit], (unsigned long long)(capsum(k, seg, n) - capsum(run_start, seg, n)));
-          run_start = k;
-          run_digit = dgt;
+      int run_start = a;
+      unsigned run_digit = 0xffffffffu;
+      for (int k0 = a; k0 < b; k0 += 8) {
+        float gv[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) gv[i] = (k0 + i < b) ? __ldg(g + k0 + i) : 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int k = k0 + i;
+          if (k < b) {
+            const unsigned dgt = (unsigned)(seg_key(gv[i], k, h, N) >> shift) & 255u;
+            if (dgt != run_digit) {
+              if (run_digit != 0xffffffffu)
+                atomicAdd(&hist[run_digit], (unsigned long long)(capsum(k, seg, n) - capsum(run_start, seg, n)));
+              run_start = k;
+              run_digit = dgt;
+            }
+          }
         }
       }
-      atomicAdd(&hist[run_digit], (unsigned long long)(capsum(r, seg, n) - capsum(run_start, seg, n)));
+      atomicAdd(&hist[run_digit], (unsigned long long)(capsum(b, seg, n) - capsum(run_start, seg, n)));
     }
     __syncthreads();
     if (tid < 32) {
@@ -188,27 +211,38 @@ __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __r
       for (int h = tid; h < N; h += kGreedyThreads) lo[h] = hi[h];
       break;
     }
+    // bytes are non-decreasing in k, so counting the active segments below / up to the chosen
+    // byte gives the narrowed range
     const unsigned D = (unsigned)sh_digit;
-    for (int h = tid; h < N; h += kGreedyThreads) {
-      int l = lo[h], r = hi[h];
-      if (l >= r) continue;
+    for (int h = tid / tph; h < N; h += heads_per_iter) {
+      const int l = lo[h], r = hi[h];
+      const int len = r - l;
+      const int a = l + (int)(((long long)len * sub) / tph), b = l + (int)(((long long)len * (sub + 1)) / tph);
+      if (a >= b) continue;
       const float* g = gains + (size_t)h * G1;
-      // digits are non-decreasing in k: binary searches for the first digit >= D and > D
-      int a = l, b = r;
-      while (a < b) {
-        const int mid = (a + b) >> 1;
-        const unsigned dgt = (unsigned)(seg_key(__ldg(g + mid), mid, h, N) >> shift) & 255u;
-        if (dgt < D) a = mid + 1; else b = mid;
+      int lt = 0, le = 0;
+      for (int k0 = a; k0 < b; k0 += 8) {
+        float gv[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) gv[i] = (k0 + i < b) ? __ldg(g + k0 + i) : 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int k = k0 + i;
+          if (k < b) {
+            const unsigned dgt = (unsigned)(seg_key(gv[i], k, h, N) >> shift) & 255u;
+            lt += dgt < D;
+            le += dgt <= D;
+          }
+        }
       }
-      const int nl = a;
-      b = r;
-      while (a < b) {
-        const int mid = (a + b) >> 1;
-        const unsigned dgt = (unsigned)(seg_key(__ldg(g + mid), mid, h, N) >> shift) & 255u;
-        if (dgt <= D) a = mid + 1; else b = mid;
-      }
-      lo[h] = nl;
-      hi[h] = a;
+      if (lt) atomicAdd(&cnt_lt[h], lt);
+      if (le) atomicAdd(&cnt_le[h], le);
+    }
+    __syncthreads();
+    for (int h = tid; h < N; h += kGreedyThreads) {
+      const int l = lo[h];
+      lo[h] = l + cnt_lt[h];
+      hi[h] = l + cnt_le[h];
     }
     __syncthreads();
   }
@@ -249,17 +283,19 @@ __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __r
 cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, float* gains,
                             int32_t* budgets, int32_t* offsets, LaunchCtx& lc) {
   cudaStream_t st = lc.st;
-  // hull: as many heads per block as fit in ~200 KB of shared memory, at most 32
-  int hb = (int)((200u * 1024u) / ((size_t)dm.P * 8u));
-  hb = hb > 32 ? 32 : (hb < 1 ? 1 : hb);
-  const size_t hull_smem = (size_t)dm.P * hb * 8;
+  // hull: one warp per head, up to 4 warps per block (3 arrays of P words per warp)
+  int hw = (int)((200u * 1024u) / ((size_t)dm.P * 12u));
+  hw = hw > 4 ? 4 : (hw < 1 ? 1 : hw);
+  const size_t hull_smem = (size_t)dm.P * hw * 12;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(hull_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hull_smem)) != cudaSuccess)
     return e;
-  hull_kernel<<<(dm.N + hb - 1) / hb, 128, hull_smem, st>>>(curves, gains, dm.N, dm.P, hb);
+  hull_kernel<<<(dm.N + hw - 1) / hw, hw * 32, hull_smem, st>>>(curves, gains, dm.N, dm.P);
   lc.mark("hull");
 
-  const size_t greedy_smem = (size_t)dm.N * 2 * sizeof(int);
+  const size_t greedy_smem = (size_t)dm.N * 4 * sizeof(int);
+  int tph = 1;  // threads per head: the largest power of two <= 1024/N, at most 32
+  while (tph < 32 && tph * 2 * dm.N <= kGreedyThreads) tph *= 2;
   if ((e = cudaFuncSetAttribute(greedy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)greedy_smem)) != cudaSuccess)
     return e;
   long long base = 0;
@@ -277,7 +313,7 @@ cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* 
     }
     args.seq0 = q0;
     greedy_kernel<<<cnt, kGreedyThreads, greedy_smem, st>>>(gains, args, budgets, offsets, dm.N, dm.P, dm.seg, dm.nseg,
-                                                            dm.n, dm.w);
+                                                            dm.n, dm.w, tph);
     lc.mark("greedy");
   }
   return cudaGetLastError();

@@ -11,7 +11,8 @@
 namespace lukv {
 namespace {
 
-constexpr int kSelThreads = 1024;
+constexpr int kSelThreads = 512;
+constexpr int kSelWarps = kSelThreads / 32;
 
 // Order-preserving map float -> uint32 (larger float <=> larger key).
 __device__ __forceinline__ uint32_t score_key(float x) {
@@ -27,25 +28,27 @@ __device__ __forceinline__ int block_sum(int v, int* buf) {
   __syncthreads();
   int total = 0;
 #pragma unroll
-  for (int i = 0; i < kSelThreads / 32; i += 4) {
+  for (int i = 0; i < kSelWarps; i += 4) {
     const int4 t = *reinterpret_cast<const int4*>(buf + i);
     total += t.x + t.y + t.z + t.w;
   }
   return total;
 }
 
-// EPT > 0: the thread keeps its EPT consecutive keys in registers (n <= 1024*EPT).
-// EPT == 0: the thread re-reads its span of `per` consecutive scores from memory in every
-// round (long contexts).
+// One CTA per head.  Warp wv owns the positions [wv*span, (wv+1)*span) and lane l of it the
+// positions wv*span + e*32 + l, so loads are coalesced and position order is (warp, e, lane).
+// EPT > 0: span = 32*EPT and the thread keeps its EPT keys in registers (n <= 512*EPT).
+// EPT == 0: span is a multiple of 32 given by the host and the keys are re-read from memory
+// in every round (long contexts).
 template <int EPT>
-__global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ pooled,
-                                                             const int32_t* __restrict__ budgets,
-                                                             const int32_t* __restrict__ offsets,
-                                                             int32_t* __restrict__ kept_idx, long long rows_cap, int n,
-                                                             int w, int per) {
-  __shared__ __align__(16) int cnt_buf[2][kSelThreads / 32];
-  __shared__ int scan_gt[kSelThreads / 32], scan_eq[kSelThreads / 32];
-  const int u = blockIdx.x, tid = threadIdx.x;
+__global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __restrict__ pooled,
+                                                                const int32_t* __restrict__ budgets,
+                                                                const int32_t* __restrict__ offsets,
+                                                                int32_t* __restrict__ kept_idx, long long rows_cap,
+                                                                int n, int w, int span_rt) {
+  __shared__ __align__(16) int cnt_buf[2][kSelWarps];
+  __shared__ int scan_gt[kSelWarps], scan_eq[kSelWarps];
+  const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
   const int b = budgets[u];
   const long long off = offsets[u];
   const float* src = pooled + (size_t)u * n;
@@ -57,14 +60,17 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
     if (b + t < room) out[b + t] = n + t;
   if (b <= 0) return;
 
-  const int span = EPT > 0 ? EPT : per;
-  const int j0 = tid * span;
+  const int span = EPT > 0 ? 32 * EPT : span_rt;
+  const int base = wv * span + lane;
+  const int iters = span >> 5;
   uint32_t keys[EPT > 0 ? EPT : 1];
   if (EPT > 0) {
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) keys[e] = (j0 + e < n) ? score_key(src[j0 + e]) : 0u;
+    for (int e = 0; e < EPT; ++e) {
+      const int j = base + 32 * e;
+      keys[e] = j < n ? score_key(src[j]) : 0u;
+    }
   }
-  const int j_end = min(n, j0 + span);
 
   // b-th largest key: largest thr with count(key >= thr) >= b.  Positions beyond n carry
   // key 0 and are never counted because every candidate is non-zero.
@@ -77,13 +83,16 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
 #pragma unroll
       for (int e = 0; e < EPT; ++e) c += keys[e] >= cand;
     } else {
-      for (int j = j0; j < j_end; ++j) c += score_key(src[j]) >= cand;
+      for (int e = 0; e < iters; ++e) {
+        const int j = base + 32 * e;
+        if (j < n) c += score_key(src[j]) >= cand;
+      }
     }
     if (block_sum(c, cnt_buf[phase]) >= b) thr = cand;
     phase ^= 1;
   }
 
-  // emit in ascending position: all keys > thr, and the first k_eq keys == thr
+  // per-warp totals of keys above / equal to the threshold, then an exclusive scan over warps
   int my_gt = 0, my_eq = 0;
   if (EPT > 0) {
 #pragma unroll
@@ -92,59 +101,51 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
       my_eq += keys[e] == thr;
     }
   } else {
-    for (int j = j0; j < j_end; ++j) {
-      const uint32_t key = score_key(src[j]);
+    for (int e = 0; e < iters; ++e) {
+      const int j = base + 32 * e;
+      const uint32_t key = j < n ? score_key(src[j]) : 0u;
       my_gt += key > thr;
       my_eq += key == thr;
     }
   }
-  // exclusive scans over the threads (thread order == position order)
-  int inc_gt = my_gt, inc_eq = my_eq;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int a = __shfl_up_sync(0xffffffffu, inc_gt, o);
-    const int c = __shfl_up_sync(0xffffffffu, inc_eq, o);
-    if ((tid & 31) >= o) {
-      inc_gt += a;
-      inc_eq += c;
-    }
-  }
-  if ((tid & 31) == 31) {
-    scan_gt[tid >> 5] = inc_gt;
-    scan_eq[tid >> 5] = inc_eq;
+  my_gt = __reduce_add_sync(0xffffffffu, my_gt);
+  my_eq = __reduce_add_sync(0xffffffffu, my_eq);
+  if (lane == 0) {
+    scan_gt[wv] = my_gt;
+    scan_eq[wv] = my_eq;
   }
   __syncthreads();
-  int before_gt = inc_gt - my_gt, before_eq = inc_eq - my_eq, total_gt = 0;
-  for (int wv = 0; wv < kSelThreads / 32; ++wv) {
-    if (wv < (tid >> 5)) {
-      before_gt += scan_gt[wv];
-      before_eq += scan_eq[wv];
+  int run_gt = 0, run_eq = 0, total_gt = 0;
+  for (int x = 0; x < kSelWarps; ++x) {
+    if (x < wv) {
+      run_gt += scan_gt[x];
+      run_eq += scan_eq[x];
     }
-    total_gt += scan_gt[wv];
+    total_gt += scan_gt[x];
   }
   const int k_eq = b - total_gt;  // ties to keep (>= 1)
+
+  // emit in ascending position: all keys > thr, and the first k_eq keys == thr
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  auto emit = [&](uint32_t key, int j) {
+    const bool gt = key > thr, eq = key == thr;
+    const uint32_t m_gt = __ballot_sync(0xffffffffu, gt), m_eq = __ballot_sync(0xffffffffu, eq);
+    const int before_gt = run_gt + __popc(m_gt & lt_mask);
+    const int before_eq = run_eq + __popc(m_eq & lt_mask);
+    if (gt || (eq && before_eq < k_eq)) {
+      const int pos = before_gt + min(before_eq, k_eq);
+      if (pos < room) out[pos] = j;
+    }
+    run_gt += __popc(m_gt);
+    run_eq += __popc(m_eq);
+  };
   if (EPT > 0) {
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) {
-      const uint32_t key = keys[e];
-      const bool gt = key > thr, eq = key == thr;
-      if (gt || (eq && before_eq < k_eq)) {
-        const int pos = before_gt + min(before_eq, k_eq);
-        if (pos < room) out[pos] = j0 + e;
-      }
-      before_gt += gt;
-      before_eq += eq;
-    }
+    for (int e = 0; e < EPT; ++e) emit(keys[e], base + 32 * e);
   } else {
-    for (int j = j0; j < j_end; ++j) {
-      const uint32_t key = score_key(src[j]);
-      const bool gt = key > thr, eq = key == thr;
-      if (gt || (eq && before_eq < k_eq)) {
-        const int pos = before_gt + min(before_eq, k_eq);
-        if (pos < room) out[pos] = j;
-      }
-      before_gt += gt;
-      before_eq += eq;
+    for (int e = 0; e < iters; ++e) {
+      const int j = base + 32 * e;
+      emit(j < n ? score_key(src[j]) : 0u, j);
     }
   }
 }
@@ -229,14 +230,16 @@ cudaError_t launch_select(const Dims& dm, const float* scores, bool scores_are_r
   const unsigned grid = (unsigned)dm.heads();
   const int n = dm.n;
   if (n <= kSelThreads * 4)
-    select_kernel<4><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 4);
+    select_kernel<4><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0);
   else if (n <= kSelThreads * 16)
-    select_kernel<16><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 16);
-  else if (n <= kSelThreads * 32)
-    select_kernel<32><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 32);
-  else
-    select_kernel<0><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w,
-                                                   (n + kSelThreads - 1) / kSelThreads);
+    select_kernel<16><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0);
+  else if (n <= kSelThreads * 64)
+    select_kernel<64><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0);
+  else {
+    const int per_warp = (n + kSelWarps - 1) / kSelWarps;
+    const int span = (per_warp + 31) & ~31;
+    select_kernel<0><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, span);
+  }
   lc.mark("select");
   return cudaGetLastError();
 }
