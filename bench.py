@@ -38,6 +38,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_32k")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="override the workload's layer count (a reduced case for profiler captures)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-heads", type=int, default=24, help="heads in the CPU-baseline sample")
     ap.add_argument("--no-e2e", action="store_true")
@@ -84,7 +86,7 @@ def run_reference(args):
     from oracle import lukv_oracle as O
     from paper_2602_08585_b200 import synth
     O.build()
-    wl = synth.CONFIGS[args.workload]
+    wl = pick_workload(args)
     heads = max(1, min(4, wl.S * wl.N))
     for _ in range(args.warmup):
         oracle_sample_seconds(wl, 1)
@@ -218,7 +220,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     lukv.lib()
 
-    wl = synth.CONFIGS[args.workload]
+    wl = pick_workload(args)
     p = lukv.make_params(wl.S, wl.L, wl.H, wl.G, wl.d, wl.T, wl.w, wl.kp, wl.dtype, wl.P)
     q, k, v = synth.gen_tensors(wl, "cuda")
     curves_np = synth.gen_curves(wl)
@@ -351,6 +353,14 @@ def run_ours(args):
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def pick_workload(args):
+    from paper_2602_08585_b200 import synth
+    wl = synth.CONFIGS[args.workload]
+    if args.layers > 0 and args.layers != wl.L:
+        wl = synth.scaled(wl, L=args.layers, name=f"{wl.name}[layers={args.layers}]")
+    return wl
 
 
 def main():
