@@ -25,9 +25,12 @@ Workspace carve_workspace(const Dims& dm, void* base) {
   const size_t heads = (size_t)dm.heads();
   ws.raw = static_cast<float*>(take(heads * dm.n * sizeof(float)));
   ws.pooled = static_cast<float*>(take(heads * dm.n * sizeof(float)));
-  ws.stats = static_cast<float*>(take(heads * score_chunks(dm) * dm.M * 2 * sizeof(float)));
+  const size_t stats_simt = heads * score_chunks(dm) * dm.M * 2 * sizeof(float);
+  const size_t stats_tc = score_tc_stats_bytes(dm);
+  ws.stats = static_cast<float*>(take(stats_simt > stats_tc ? stats_simt : stats_tc));
   ws.lse = static_cast<float*>(take(heads * dm.M * sizeof(float)));
   ws.gains = static_cast<float*>(take((size_t)dm.N * (dm.P - 1) * sizeof(float)));
+  ws.head_flags = static_cast<int*>(take(score_tc_flag_bytes(dm)));
   ws.bytes = off;
   return ws;
 }

@@ -3,6 +3,7 @@
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 
 #include "lukv.h"
@@ -26,13 +27,17 @@ struct Dims {
 struct Workspace {
   float* raw;        // [S*N][n]   un-pooled scores
   float* pooled;     // [S*N][n]   pooled scores (fused path)
-  float* stats;      // [S*N][chunks][M][2] partial (max, sum) of the SIMT scorer
+  float* stats;      // partial (reference, sum-exp) per row: [S*N][chunks][M][2] (FP32-pipe scorer) or
+                     // [S*N][items][256][2] (tensor-core scorer)
   float* lse;        // [S*N][M]   row log-sum-exp in the exp2 domain
   float* gains;      // [N][P-1]   hull gains
+  int* head_flags;   // tensor-core scorer: [S*N] items delivered per head, then the (lse, tag) rows
   size_t bytes;
 };
 
 int score_chunks(const Dims& dm);                       // key chunks per head of the SIMT scorer
+size_t score_tc_stats_bytes(const Dims& dm);            // pass-1 partials of the tensor-core scorer
+size_t score_tc_flag_bytes(const Dims& dm);             // its zero-initialised counters and (lse, tag) rows
 Workspace carve_workspace(const Dims& dm, void* base);  // base may be null (size query)
 
 // Launch bookkeeping: counts the kernels a call enqueues and, when a timeline is attached

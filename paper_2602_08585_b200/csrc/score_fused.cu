@@ -1,0 +1,873 @@
+// Stage (a) on the 5th-generation tensor cores (bf16, head_dim 128): one persistent kernel
+// computes the un-pooled observation-window scores of every head.
+//
+// The window logits S = Q K^T of Eq. 1 (Sec. 3.1) come from tcgen05.mma with fp32
+// accumulators in tensor memory; operands are staged in shared memory by TMA (128-byte
+// swizzle, no multicast).  A row's softmax normaliser needs every key of the head before any
+// probability is final, so each head is swept twice:
+//   pass 1  D[query row][key]: a thread owns one query row in TMEM and folds its columns into
+//           a (reference, sum-exp) pair; the partials of a work item go to global memory and
+//           the CTA that delivers a head's last partial folds them into the row log-sum-exp
+//   pass 2  D[key][query row] (operands swapped): a thread owns one key and adds
+//           exp2(x - lse_row) over all rows in registers -> the un-pooled score of the key
+// Both operand tiles are K-major, so the same shared-memory tiles serve as A or B.
+//
+// Work item = (head, run of item_tiles key tiles).  Items are dealt round-robin to a grid of
+// at most one CTA per SM, launched cooperatively (all CTAs resident).  A CTA runs pass 1
+// lag-1 items ahead of pass 2, so that the log-sum-exp of a head is normally complete before
+// pass 2 needs it, and the key tiles pass 2 re-reads are still in L2: K crosses HBM once.
+//
+// Warp roles per CTA: 4*NQ epilogue warps in NQ quads (a warp may only read the TMEM lanes
+// 32*(warp%4)..+31), then one warp each: TMA producer, MMA issuer and TMEM owner, publisher
+// (pass-1 partials -> global memory, head completion), prefetcher (-lse -> shared memory).
+// The last two keep every global-memory round trip off the epilogue warps.
+// Every wait is bounded; a wait that runs out raises the CTA's abort flag and stores
+// LUKV_ERR_TIMEOUT to the status word; the CTA then skips the remaining work and tears down
+// normally.
+#include <cuda.h>
+#include <stdlib.h>
+
+#include "common.cuh"
+
+namespace lukv {
+namespace {
+
+constexpr int kTileKeys = 128;               // keys per shared-memory stage / per MMA M or N
+constexpr int kHalfBytes = kTileKeys * 128;  // one 64-channel half of a 128-row tile (SW128 atom rows)
+constexpr int kStageBytes = 2 * kHalfBytes;  // 128 keys x 128 channels bf16
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kMaxLag = 6;                   // a CTA runs pass 1 at most this many items ahead of pass 2
+constexpr int kFinBytes = 16384;             // one block of partials folded by a head's last item
+
+// ---- PTX wrappers ------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Raises the CTA's abort flag and reports the timeout.
+__device__ __forceinline__ void raise_abort(volatile int* abort_flag, int32_t* dev_status) {
+  *abort_flag = 1;
+  if (dev_status) atomicExch(dev_status, (int32_t)LUKV_ERR_TIMEOUT);
+}
+// Bounded wait: false when the CTA is aborting or the limit is reached (then it raises the abort).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
+  if (*abort_flag) return false;
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (i > 4096) __nanosleep(128);
+  }
+  raise_abort(abort_flag, dev_status);
+  return false;
+}
+
+__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
+  int old;
+  asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
+// 8-byte load that always observes memory at GPU scope (used to poll data another CTA writes)
+__device__ __forceinline__ float2 ld_relaxed_f2(const float2* p) {
+  float2 v;
+  asm volatile("ld.relaxed.gpu.global.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
+  return v;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy)
+      : "memory");
+}
+// untiled bulk copy global -> shared (16-byte aligned addresses, size a multiple of 16)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulation; issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"((uint32_t)accumulate)
+      : "memory");
+}
+// mbarrier arrives once every tcgen05.mma issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp gets TMEM lane (base lane + i).
+// The load is asynchronous: the registers are valid only after tmem_ld_wait on the same array.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+// Waits for every outstanding tcgen05.ld of this thread.  The array is passed as an in/out
+// operand so that no use of its registers can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(float (&v)[32]) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]),
+                 "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]),
+                 "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the
+// 128-byte swizzle (8-row groups 1024 bytes apart), as written by TMA.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  return (uint64_t)((saddr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// Packed pairs of fp32 (one 64-bit register): two lanes per FMA-pipe instruction.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t p, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(p));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// both lanes of a packed pair through exp2
+__device__ __forceinline__ uint64_t ex2_pair(uint64_t x) {
+  float a, b;
+  unpack2(x, a, b);
+  return pack2(ex2(a), ex2(b));
+}
+__device__ __forceinline__ float sum4(uint64_t p, uint64_t q) {
+  float a, b, c, d;
+  unpack2(p, a, b);
+  unpack2(q, c, d);
+  return (a + b) + (c + d);
+}
+
+// ---- shared-memory layout ---------------------------------------------------------------------
+
+template <int MT, int NQ>
+struct Plan {
+  static_assert(MT == 1 || NQ == 2, "two query-row blocks are split over exactly two quads");
+  static constexpr int kEpiWarps = 4 * NQ;
+  static constexpr int kThreads = (kEpiWarps + 4) * 32;  // + TMA producer, MMA issuer, publisher, prefetcher
+  static constexpr int kStages = MT == 1 ? 3 : 2;      // key-tile ring
+  static constexpr int kQSlots = 2;                    // query tiles of the job in the tensor pipe and the next one
+  static constexpr int kQBytes = MT * kStageBytes;     // [half][MT*128 rows][128 B]
+  static constexpr int kFinBufs = MT == 1 ? 2 : 1;     // blocks of partials in flight while a head is folded
+  static constexpr int kFinParts = kFinBytes / (128 * MT * 8);  // partials per block
+  static constexpr int kKOff = kQSlots * kQBytes;
+  static constexpr int kFinOff = kKOff + kStages * kStageBytes;
+  static constexpr int kBarOff = kFinOff + kFinBufs * kFinBytes;
+  static constexpr int kNumBufs = 4 / MT;              // accumulator buffers in TMEM
+  static constexpr int kBufCols = 128 * MT;
+  // barriers: full[kStages], empty[kStages], qfull[kQSlots], qempty[kQSlots], tfull[kNumBufs],
+  // tempty[kNumBufs], pub_full[NQ], pub_empty[NQ], lse_full[kMaxLag], lse_empty[kMaxLag], fin[kFinBufs]
+  static constexpr int kBarFull = 0, kBarEmpty = kStages, kBarQFull = 2 * kStages, kBarQEmpty = kBarQFull + kQSlots,
+                       kBarTFull = kBarQEmpty + kQSlots, kBarTEmpty = kBarTFull + kNumBufs,
+                       kBarPubFull = kBarTEmpty + kNumBufs, kBarPubEmpty = kBarPubFull + NQ,
+                       kBarLseFull = kBarPubEmpty + NQ, kBarLseEmpty = kBarLseFull + kMaxLag,
+                       kBarFin = kBarLseEmpty + kMaxLag, kNumBars = kBarFin + kFinBufs;
+  static constexpr int kMiscOff = (kBarOff + kNumBars * 8 + 15) & ~15;  // tmem base, abort flag
+  static constexpr int kPubOff = kMiscOff + 16;        // [NQ][128] (reference, sum-exp) handed to the publisher warp
+  static constexpr int kLseOff = kPubOff + NQ * 128 * 8;  // [kMaxLag][256] -lse of the pass-2 jobs to come
+  static_assert(kLseOff % 16 == 0, "lse rows are read with 16-byte loads");
+  static constexpr int kTotal = kLseOff + kMaxLag * 256 * 4 + 1024;  // + slack for the 1024-byte alignment
+  static_assert(kTotal <= 232448, "exceeds the shared memory of one CTA");
+};
+
+struct FusedArgs {
+  float* stats;        // pass 1 partials: [heads][items_per_head][128*MT] (reference, sum-exp), exp2 domain
+  float* lse;          // [heads][lse_rows] (row log-sum-exp in the exp2 domain, tag); zero at launch
+  float* raw;          // pass 2 out: [heads][n]
+  int* head_cnt;       // [heads] items whose partials were delivered (zero at launch)
+  int32_t* dev_status;
+  int M, T, w, n;
+  int lse_rows;        // M rounded up to a multiple of 2
+  int head0, nheads;   // heads [head0, head0+nheads) are scored by this launch
+  int item_tiles, items_per_head, tiles_T, tiles_n;
+  int npad;            // pass 2: query rows rounded up to a multiple of 32 (MMA N and columns read)
+  int lag;             // 2..kMaxLag: pass 1 of item k+lag-1 precedes pass 2 of item k
+  int l2_hints;        // 1: pass-1 key loads ask L2 to keep the lines, pass-2 loads to drop them first
+  float scale_log2;
+};
+
+struct Job {
+  int u;       // head
+  int c;       // item of the head
+  int tile0;   // first key tile
+  int ntiles;  // key tiles of this job (may be 0)
+  bool p2;
+};
+
+__device__ __forceinline__ Job make_job(int k, bool p2, const FusedArgs& a) {
+  Job j;
+  j.p2 = p2;
+  const int item = (int)blockIdx.x + k * (int)gridDim.x;
+  const int hu = item / a.items_per_head;
+  j.c = item - hu * a.items_per_head;
+  j.u = a.head0 + hu;
+  j.tile0 = j.c * a.item_tiles;
+  const int lim = p2 ? a.tiles_n : a.tiles_T;
+  j.ntiles = max(0, min(a.item_tiles, lim - j.tile0));
+  return j;
+}
+
+// Job `idx` of a CTA that owns K items: lag-1 pass-1 jobs first, then pass 1 of item k+lag-1
+// alternating with pass 2 of item k, then the remaining pass-2 jobs.
+__device__ __forceinline__ Job decode_job(int idx, int K, const FusedArgs& a) {
+  const int lead = min(a.lag - 1, K);
+  if (idx < lead) return make_job(idx, false, a);
+  const int r = idx - lead, pairs = 2 * (K - lead);
+  if (r < pairs) return (r & 1) ? make_job(r >> 1, true, a) : make_job(lead + (r >> 1), false, a);
+  return make_job(K - lead + (r - pairs), true, a);
+}
+
+// Pass 1, 32 columns (keys jbase..jbase+31) of one query row: fold into the running (m, l).
+// (m, l) means sum over the keys seen so far of exp2(x - m); m is a reference point, not
+// necessarily the maximum: the common path adds the new terms relative to the current m and
+// only re-references (exactly, from the chunk maximum) when the chunk sum leaves a safe range
+// -- which also covers the first chunk (m = -inf) and any overflow.
+template <bool MASKED>
+__device__ __forceinline__ void p1_chunk(const float (&v)[32], int jbase, int lim, float scale_log2, float& m,
+                                         float& l) {
+  float x[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) x[i] = (!MASKED || jbase + i <= lim) ? v[i] : -INFINITY;
+  const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m, -m);
+  uint64_t acc0 = 0ull, acc1 = 0ull;  // bit pattern of (+0, +0)
+#pragma unroll
+  for (int i = 0; i < 32; i += 4) {
+    acc0 = fadd2(acc0, ex2_pair(ffma2(pack2(x[i], x[i + 1]), sc2, nm2)));
+    acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(x[i + 2], x[i + 3]), sc2, nm2)));
+  }
+  const float cs = sum4(acc0, acc1);
+  if (cs <= 1e12f) {  // false for inf and NaN
+    l += cs;
+    return;
+  }
+  float cmax = x[0];
+#pragma unroll
+  for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, x[i]);
+  if (cmax == -INFINITY) return;  // every key of the chunk is masked
+  const float mn = fmaxf(m, cmax * scale_log2);  // scale > 0
+  float a0 = l * ex2(m - mn), a1 = 0.f;
+#pragma unroll
+  for (int i = 0; i < 32; i += 2) {
+    a0 += ex2(fmaf(x[i], scale_log2, -mn));
+    a1 += ex2(fmaf(x[i + 1], scale_log2, -mn));
+  }
+  l = a0 + a1;
+  m = mn;
+}
+
+// Pass 2, 32 columns (query rows c0..c0+31) of one key: add the probabilities.
+__device__ __forceinline__ void p2_chunk(const float (&v)[32], const float* nlse, uint64_t sc2, uint64_t& acc0,
+                                         uint64_t& acc1) {
+#pragma unroll
+  for (int i = 0; i < 32; i += 4) {
+    const ulonglong2 ls = *reinterpret_cast<const ulonglong2*>(nlse + i);  // (-lse[i], -lse[i+1]), (-lse[i+2], -lse[i+3])
+    acc0 = fadd2(acc0, ex2_pair(ffma2(pack2(v[i], v[i + 1]), sc2, ls.x)));
+    acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(v[i + 2], v[i + 3]), sc2, ls.y)));
+  }
+}
+
+template <int MT, int NQ>
+__global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
+    score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
+                       const FusedArgs a) {
+  using P = Plan<MT, NQ>;
+  constexpr int kStages = P::kStages;
+  constexpr int kNumBufs = P::kNumBufs;
+  constexpr int kEpiWarps = P::kEpiWarps;
+  constexpr int kRowsPad = 128 * MT;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t q_s = sbase;
+  const uint32_t k_s = sbase + P::kKOff;
+  const uint32_t bars = sbase + P::kBarOff;
+  auto bar = [&](int first, int i) { return bars + 8u * (uint32_t)(first + i); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + P::kMiscOff);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + P::kMiscOff + 4);
+  float2* pub_s = reinterpret_cast<float2*>(smem + P::kPubOff);   // [NQ][128]
+  float* nlse_s = reinterpret_cast<float*>(smem + P::kLseOff);    // [kMaxLag][256]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_items = a.nheads * a.items_per_head;
+  const int K = (total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // items of this CTA (>= 1)
+  const int njobs = 2 * K;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar(P::kBarFull, s), 1);
+      mbar_init(bar(P::kBarEmpty, s), 1);
+    }
+    for (int s = 0; s < P::kQSlots; ++s) {
+      mbar_init(bar(P::kBarQFull, s), 1);
+      mbar_init(bar(P::kBarQEmpty, s), 1);
+    }
+    for (int b = 0; b < kNumBufs; ++b) {
+      mbar_init(bar(P::kBarTFull, b), 1);
+      mbar_init(bar(P::kBarTEmpty, b), MT == 2 ? 8 : 4);
+    }
+    for (int q = 0; q < NQ; ++q) {
+      mbar_init(bar(P::kBarPubFull, q), 4);
+      mbar_init(bar(P::kBarPubEmpty, q), 1);
+    }
+    for (int s = 0; s < kMaxLag; ++s) {
+      mbar_init(bar(P::kBarLseFull, s), 1);
+      mbar_init(bar(P::kBarLseEmpty, s), kEpiWarps);
+    }
+    for (int b = 0; b < P::kFinBufs; ++b) mbar_init(bar(P::kBarFin, b), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kEpiWarps + 1) tmem_alloc(smem_u32((const void*)tmem_slot), 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == kEpiWarps) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
+      uint32_t tt = 0, jq = 0;
+      for (int idx = 0; idx < njobs; ++idx) {
+        const Job j = decode_job(idx, K, a);
+        if (j.ntiles == 0) continue;
+        const uint32_t slot = jq % P::kQSlots;
+        if (!mbar_wait(bar(P::kBarQEmpty, slot), ((jq / P::kQSlots) & 1) ^ 1, abort_flag, a.dev_status)) break;
+        mbar_expect_tx(bar(P::kBarQFull, slot), P::kQBytes);
+        const uint32_t qd = q_s + slot * P::kQBytes;
+        for (int h = 0; h < 2; ++h)
+          for (int mt = 0; mt < MT; ++mt) {
+            const uint32_t dst = qd + h * (MT * kHalfBytes) + mt * kHalfBytes;
+            if (a.l2_hints) tma_load_2d_hint(dst, &q_map, bar(P::kBarQFull, slot), h * 64, j.u * a.M + mt * 128, keep);
+            else tma_load_2d(dst, &q_map, bar(P::kBarQFull, slot), h * 64, j.u * a.M + mt * 128);
+          }
+        ++jq;
+        bool ok = true;
+        for (int t = 0; t < j.ntiles; ++t, ++tt) {
+          const uint32_t s = tt % kStages, ph = (tt / kStages) & 1;
+          if (!(ok = mbar_wait(bar(P::kBarEmpty, s), ph ^ 1, abort_flag, a.dev_status))) break;
+          mbar_expect_tx(bar(P::kBarFull, s), kStageBytes);
+          const int row = j.u * a.T + (j.tile0 + t) * kTileKeys;
+          const uint32_t dst = k_s + s * kStageBytes;
+          if (a.l2_hints) {
+            const uint64_t pol = j.p2 ? drop : keep;
+            tma_load_2d_hint(dst, &k_map, bar(P::kBarFull, s), 0, row, pol);
+            tma_load_2d_hint(dst + kHalfBytes, &k_map, bar(P::kBarFull, s), 64, row, pol);
+          } else {
+            tma_load_2d(dst, &k_map, bar(P::kBarFull, s), 0, row);
+            tma_load_2d(dst + kHalfBytes, &k_map, bar(P::kBarFull, s), 64, row);
+          }
+        }
+        if (!ok) break;
+      }
+    }
+  } else if (warp == kEpiWarps + 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      uint32_t tt = 0, jq = 0;
+      for (int idx = 0; idx < njobs; ++idx) {
+        const Job j = decode_job(idx, K, a);
+        if (j.ntiles == 0) continue;
+        const uint32_t slot = jq % P::kQSlots;
+        if (!mbar_wait(bar(P::kBarQFull, slot), (jq / P::kQSlots) & 1, abort_flag, a.dev_status)) break;
+        const uint32_t qd = q_s + slot * P::kQBytes;
+        bool ok = true;
+        for (int t = 0; t < j.ntiles; ++t, ++tt) {
+          const uint32_t s = tt % kStages, ph = (tt / kStages) & 1;
+          const uint32_t buf = tt % kNumBufs, use = tt / kNumBufs;
+          if (!(ok = mbar_wait(bar(P::kBarTEmpty, buf), (use & 1) ^ 1, abort_flag, a.dev_status))) break;
+          if (!(ok = mbar_wait(bar(P::kBarFull, s), ph, abort_flag, a.dev_status))) break;
+          tc_fence_after();
+          const uint32_t kt = k_s + s * kStageBytes;
+          const uint32_t d_tmem = tmem_base + buf * P::kBufCols;
+          if (!j.p2) {
+            // D[q row][key]: A = Q (M-tile mt), B = K tile
+            constexpr uint32_t idesc = instr_desc_bf16(128, kTileKeys);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks) {
+                const int h = ks >> 2, sub = ks & 3;
+                const uint64_t da = smem_desc_sw128(qd + h * (MT * kHalfBytes) + mt * kHalfBytes) + (uint64_t)(sub * 2);
+                const uint64_t db = smem_desc_sw128(kt + h * kHalfBytes) + (uint64_t)(sub * 2);
+                umma_bf16(d_tmem + mt * 128, da, db, idesc, ks > 0);
+              }
+          } else {
+            // D[key][q row]: A = K tile, B = Q (npad rows)
+            const uint32_t idesc = instr_desc_bf16(128, a.npad);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const int h = ks >> 2, sub = ks & 3;
+              const uint64_t da = smem_desc_sw128(kt + h * kHalfBytes) + (uint64_t)(sub * 2);
+              const uint64_t db = smem_desc_sw128(qd + h * (MT * kHalfBytes)) + (uint64_t)(sub * 2);
+              umma_bf16(d_tmem, da, db, idesc, ks > 0);
+            }
+          }
+          umma_commit(bar(P::kBarEmpty, s));     // the stage may be refilled once these MMAs have read it
+          umma_commit(bar(P::kBarTFull, buf));   // the accumulator is complete
+        }
+        if (!ok) break;
+        umma_commit(bar(P::kBarQEmpty, slot));   // the query tiles may be replaced
+        ++jq;
+      }
+    }
+  } else if (warp == kEpiWarps + 2) {
+    // ---------------- publisher: pass-1 partials -> global memory, head completion ----------------
+    // For item k: merge the quads' partials, store them, count the item in (release).  The warp
+    // that counts a head's last item folds all its partials into the row log-sum-exp and stores
+    // it as (value, tag) pairs, which the prefetchers of the head's CTAs poll.
+    uint32_t fin_uses[P::kFinBufs] = {};
+    for (int k = 0; k < K; ++k) {
+      const Job j1 = make_job(k, false, a);
+      bool ok = true;
+      for (int q = 0; q < NQ; ++q) ok = mbar_wait(bar(P::kBarPubFull, q), k & 1, abort_flag, a.dev_status) && ok;
+      if (ok) {
+        float2* dst = reinterpret_cast<float2*>(a.stats) + ((size_t)j1.u * a.items_per_head + j1.c) * kRowsPad;
+#pragma unroll
+        for (int rr = 0; rr < kRowsPad; rr += 32) {
+          float2 v = pub_s[rr + lane];
+          if (MT == 1) {
+            // the quads hold partials of the same 128 rows over different key tiles: merge them
+#pragma unroll
+            for (int q = 1; q < NQ; ++q) {
+              const float2 o = pub_s[q * 128 + rr + lane];
+              if (o.y > 0.f) {  // an empty partial is (-inf, 0)
+                const float mn = fmaxf(v.x, o.x);
+                v.y = v.y * ex2(v.x - mn) + o.y * ex2(o.x - mn);
+                v.x = mn;
+              }
+            }
+          }
+          dst[rr + lane] = v;  // rows beyond M carry (-inf, 0)
+        }
+      }
+      __syncwarp();
+      if (lane == 0 && ok)
+        for (int q = 0; q < NQ; ++q) mbar_arrive(bar(P::kBarPubEmpty, q), 1);
+      // count the item in (release: the partials above; acquire: everybody else's)
+      int last = 0;
+      if (lane == 0 && ok && !*abort_flag) last = atom_add_acq_rel(a.head_cnt + j1.u, 1) == a.items_per_head - 1;
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (last) {
+        // Fold the head's partials: the bulk-copy engine brings them into shared memory in blocks of
+        // kFinParts items (one round trip per block instead of one per load); every lane folds its rows.
+        constexpr int kRowsLane = 4 * MT;
+        const char* src = reinterpret_cast<const char*>(a.stats) + (size_t)j1.u * a.items_per_head * kRowsPad * 8;
+        const int nblk = (a.items_per_head + P::kFinParts - 1) / P::kFinParts;
+        auto request = [&](int blk) {  // lane 0
+          const int parts = min(P::kFinParts, a.items_per_head - blk * P::kFinParts);
+          const uint32_t bytes = (uint32_t)parts * kRowsPad * 8, b = blk % P::kFinBufs;
+          mbar_expect_tx(bar(P::kBarFin, b), bytes);
+          bulk_load(sbase + P::kFinOff + b * kFinBytes, src + (size_t)blk * P::kFinParts * kRowsPad * 8, bytes,
+                    bar(P::kBarFin, b));
+        };
+        asm volatile("fence.proxy.async;" ::: "memory");
+        if (lane == 0)
+          for (int blk = 0; blk < nblk && blk < P::kFinBufs; ++blk) request(blk);
+        float fm[kRowsLane], fl[kRowsLane];
+#pragma unroll
+        for (int jj = 0; jj < kRowsLane; ++jj) fm[jj] = -INFINITY, fl[jj] = 0.f;
+        bool fin_ok = true;
+        for (int blk = 0; blk < nblk; ++blk) {
+          const uint32_t b = blk % P::kFinBufs;
+          fin_ok = fin_ok && mbar_wait(bar(P::kBarFin, b), fin_uses[b] & 1, abort_flag, a.dev_status);
+          ++fin_uses[b];
+          if (fin_ok) {
+            const float2* part = reinterpret_cast<const float2*>(smem + P::kFinOff + b * kFinBytes);
+            const int parts = min(P::kFinParts, a.items_per_head - blk * P::kFinParts);
+            float cm[kRowsLane], cl[kRowsLane];
+#pragma unroll
+            for (int jj = 0; jj < kRowsLane; ++jj) cm[jj] = fm[jj], cl[jj] = 0.f;
+            for (int c = 0; c < parts; ++c)
+#pragma unroll
+              for (int jj = 0; jj < kRowsLane; ++jj) {
+                const float2 v = part[c * kRowsPad + 32 * jj + lane];
+                if (v.y > 0.f) cm[jj] = fmaxf(cm[jj], v.x);  // an empty partial is (-inf, 0)
+              }
+            for (int c = 0; c < parts; ++c)
+#pragma unroll
+              for (int jj = 0; jj < kRowsLane; ++jj) {
+                const float2 v = part[c * kRowsPad + 32 * jj + lane];
+                if (v.y > 0.f) cl[jj] = fmaf(v.y, ex2(v.x - cm[jj]), cl[jj]);
+              }
+#pragma unroll
+            for (int jj = 0; jj < kRowsLane; ++jj)
+              if (cl[jj] > 0.f) {
+                fl[jj] = fmaf(fl[jj], ex2(fm[jj] - cm[jj]), cl[jj]);
+                fm[jj] = cm[jj];
+              }
+          }
+          __syncwarp();
+          if (lane == 0 && fin_ok && blk + P::kFinBufs < nblk) request(blk + P::kFinBufs);
+        }
+        float2* out = reinterpret_cast<float2*>(a.lse) + (size_t)j1.u * a.lse_rows;
+#pragma unroll
+        for (int jj = 0; jj < kRowsLane; ++jj) {
+          const int row = 32 * jj + lane;
+          if (row < a.lse_rows && fin_ok) __stcg(out + row, make_float2(fm[jj] + log2f(fl[jj]), 1.f));
+        }
+      }
+    }
+  } else if (warp == kEpiWarps + 3) {
+    // ---------------- prefetcher: -lse of the pass-2 jobs to come -> shared memory ----------------
+    // The log-sum-exp rows are stored as (value, tag) pairs that are zero at launch; polling the
+    // data itself saves a flag round trip.  The quads reach pass 2 of item k several jobs after its
+    // pass 1, so this latency is normally hidden.
+    constexpr int kRowsLane = 4 * MT;
+    uint32_t p2c = 0;
+    for (int k = 0; k < K; ++k) {
+      const Job j2 = make_job(k, true, a);
+      if (j2.ntiles == 0) continue;
+      const uint32_t slot = p2c % a.lag;
+      const bool ok = mbar_wait(bar(P::kBarLseEmpty, slot), ((p2c / a.lag) & 1) ^ 1, abort_flag, a.dev_status);
+      const float2* src = reinterpret_cast<const float2*>(a.lse) + (size_t)j2.u * a.lse_rows;
+      float2 v[kRowsLane];
+      bool have = false;
+      if (ok) {
+        for (uint32_t spin = 0; spin < kSpinLimit && !have; ++spin) {
+          bool mine = true;
+#pragma unroll
+          for (int jj = 0; jj < kRowsLane; ++jj) {
+            const int row = 32 * jj + lane;
+            if (row < a.M) {
+              v[jj] = ld_relaxed_f2(src + row);
+              mine = mine && v[jj].y != 0.f;
+            }
+          }
+          have = __all_sync(0xffffffffu, mine);
+          if (!have) {
+            if (*abort_flag) break;
+            if (spin > 16) __nanosleep(200);
+          }
+        }
+        if (!have && lane == 0 && !*abort_flag) raise_abort(abort_flag, a.dev_status);
+      }
+      __syncwarp();
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) {
+        const int row = 32 * jj + lane;
+        nlse_s[slot * 256 + row] = (have && jj < kRowsLane && row < a.M) ? -v[jj < kRowsLane ? jj : 0].x : -INFINITY;
+      }
+      __syncwarp();
+      if (lane == 0 && ok) mbar_arrive(bar(P::kBarLseFull, slot), 1);
+      ++p2c;
+    }
+  } else {
+    // ---------------- epilogue quads ----------------
+    const int quad = warp >> 2;
+    const int qtid = threadIdx.x & 127;                          // TMEM lane of this thread
+    const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+    const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2);
+    uint32_t tt = 0, p1c = 0, p2c = 0;
+    for (int idx = 0; idx < njobs; ++idx) {
+      const Job j = decode_job(idx, K, a);
+      if (j.ntiles == 0) continue;
+      if (!j.p2) {
+        // ---- pass 1: (reference, sum-exp) of this thread's query row over the job's keys
+        const int r = (MT == 2 ? 128 * quad : 0) + qtid;
+        const int lim = r < a.M ? a.n + (r % a.w) : -1;           // last visible key; -1: padded row
+        float m = -INFINITY, l = 0.f;
+        for (int t = 0; t < j.ntiles; ++t, ++tt) {
+          if (MT == 1 && (int)(tt % NQ) != quad) continue;
+          const uint32_t buf = tt % kNumBufs, use = tt / kNumBufs;
+          const bool ok = mbar_wait(bar(P::kBarTFull, buf), use & 1, abort_flag, a.dev_status);
+          if (ok) {
+            tc_fence_after();
+            const int j0 = (j.tile0 + t) * kTileKeys;
+            const bool masked = j0 + kTileKeys > a.n;             // tile reaches into the window / past T
+            const uint32_t tcol = tmem_base + lane_addr + buf * P::kBufCols + (MT == 2 ? 128 * quad : 0);
+            float va[32], vb[32];
+            tmem_ld32(tcol, va);
+#pragma unroll
+            for (int c = 0; c < 4; c += 2) {
+              tmem_ld_wait(va);
+              tmem_ld32(tcol + 32 * (c + 1), vb);
+              if (lim >= 0) {
+                if (masked) p1_chunk<true>(va, j0 + 32 * c, lim, a.scale_log2, m, l);
+                else p1_chunk<false>(va, j0 + 32 * c, lim, a.scale_log2, m, l);
+              }
+              tmem_ld_wait(vb);
+              if (c + 2 < 4) tmem_ld32(tcol + 32 * (c + 2), va);
+              if (lim >= 0) {
+                if (masked) p1_chunk<true>(vb, j0 + 32 * (c + 1), lim, a.scale_log2, m, l);
+                else p1_chunk<false>(vb, j0 + 32 * (c + 1), lim, a.scale_log2, m, l);
+              }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(P::kBarTEmpty, buf), 1);
+          }
+        }
+        // hand the partial to the publisher warp
+        const bool ok = mbar_wait(bar(P::kBarPubEmpty, quad), (p1c & 1) ^ 1, abort_flag, a.dev_status);
+        if (ok) pub_s[quad * 128 + qtid] = make_float2(m, l);
+        __syncwarp();
+        if (lane == 0 && ok) mbar_arrive(bar(P::kBarPubFull, quad), 1);
+        ++p1c;
+      } else {
+        // ---- pass 2: this thread's key, summed over all query rows
+        const uint32_t slot = p2c % a.lag;
+        const bool have_lse = mbar_wait(bar(P::kBarLseFull, slot), (p2c / a.lag) & 1, abort_flag, a.dev_status);
+        const float* nlse = nlse_s + slot * 256;
+        for (int t = 0; t < j.ntiles; ++t, ++tt) {
+          if ((int)(tt % NQ) != quad) continue;
+          const uint32_t buf = tt % kNumBufs, use = tt / kNumBufs;
+          const bool ok = mbar_wait(bar(P::kBarTFull, buf), use & 1, abort_flag, a.dev_status);
+          if (ok) {
+            tc_fence_after();
+            const int key = (j.tile0 + t) * kTileKeys + qtid;
+            const uint32_t tcol = tmem_base + lane_addr + buf * P::kBufCols;
+            uint64_t acc0 = 0ull, acc1 = 0ull;
+            float va[32], vb[32];
+            tmem_ld32(tcol, va);
+#pragma unroll 1
+            for (int c0 = 0; c0 < a.npad; c0 += 64) {
+              tmem_ld_wait(va);
+              const bool two = c0 + 32 < a.npad;
+              if (two) tmem_ld32(tcol + c0 + 32, vb);
+              p2_chunk(va, nlse + c0, sc2, acc0, acc1);
+              if (two) {
+                tmem_ld_wait(vb);
+                if (c0 + 64 < a.npad) tmem_ld32(tcol + c0 + 64, va);
+                p2_chunk(vb, nlse + c0 + 32, sc2, acc0, acc1);
+              }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(P::kBarTEmpty, buf), MT == 2 ? 2 : 1);
+            if (key < a.n) a.raw[(size_t)j.u * a.n + key] = sum4(acc0, acc1);
+          }
+        }
+        __syncwarp();
+        if (lane == 0 && have_lse) mbar_arrive(bar(P::kBarLseEmpty, slot), 1);
+        ++p2c;
+      }
+    }
+  }
+
+  // ---------------- teardown ----------------
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // give copies that may still be in flight time to land before the shared memory is released
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+  }
+  if (warp == kEpiWarps + 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---- host side --------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// 2-D bf16 tensor [rows][128] with boxes of 64 channels x 128 rows, 128-byte swizzle, zero fill.
+bool make_map(CUtensorMap* map, const void* base, uint64_t rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {128, rows};
+  const cuuint64_t strides[1] = {256};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int MT, int NQ>
+cudaError_t launch_fused(const CUtensorMap& qm, const CUtensorMap& km, FusedArgs args, LaunchCtx& lc) {
+  using P = Plan<MT, NQ>;
+  const int smem = P::kTotal;
+  auto kern = score_fused_kernel<MT, NQ>;
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
+  int dev = 0, sms = 0, per_sm = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, P::kThreads, smem)) != cudaSuccess) return e;
+  if (per_sm < 1 || sms < 1) return cudaErrorLaunchOutOfResources;
+  // A CTA runs pass 1 of later items before pass 2 of the current one, so a head's items must
+  // not outnumber the CTAs (else a CTA would wait for partials that it is due to produce itself).
+  while ((args.tiles_T + args.item_tiles - 1) / args.item_tiles > sms) ++args.item_tiles;
+  args.items_per_head = (args.tiles_T + args.item_tiles - 1) / args.item_tiles;
+  const int total_items = args.nheads * args.items_per_head;
+  const int grid = total_items < sms ? total_items : sms;  // one CTA per SM: each owns the SM's tensor memory
+  void* params[] = {(void*)&qm, (void*)&km, (void*)&args};
+  // cooperative launch: the CTAs of a head wait for one another, so all must be resident
+  e = cudaLaunchCooperativeKernel((const void*)kern, dim3((unsigned)grid), dim3(P::kThreads), params, (size_t)smem,
+                                  lc.st);
+  lc.mark("score_fused");
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+int env_int(const char* name, int lo, int hi, int dflt) {
+  const char* e = getenv(name);
+  const int x = e ? atoi(e) : dflt;
+  return (e && x >= lo && x <= hi) ? x : dflt;
+}
+
+// Offset of the (lse, tag) rows inside the zero-initialised block that starts with the [heads] counters.
+size_t lse_tag_offset(const Dims& dm) { return ((size_t)dm.heads() * sizeof(int) + 255) & ~(size_t)255; }
+
+}  // namespace
+
+// Key tiles per work item (the smallest the scorer uses; it grows for very long contexts).
+// LUKV_ITEM_TILES (1..64) overrides the default for tuning runs.
+int score_item_tiles() {
+  static const int v = env_int("LUKV_ITEM_TILES", 1, 64, 8);
+  return v;
+}
+// Bytes of pass-1 partials the tensor-core scorer may write for these sizes.
+size_t score_tc_stats_bytes(const Dims& dm) {
+  const size_t tiles = ((size_t)dm.T + kTileKeys - 1) / kTileKeys;
+  const size_t items = (tiles + score_item_tiles() - 1) / score_item_tiles();
+  return (size_t)dm.heads() * items * 256 * 2 * sizeof(float);
+}
+// Bytes of the block that must be zero at launch: [heads] counters, then [heads][lse_rows][2] floats.
+size_t score_tc_flag_bytes(const Dims& dm) {
+  return lse_tag_offset(dm) + (size_t)dm.heads() * ((dm.M + 1) & ~1) * 2 * sizeof(float);
+}
+
+bool score_tc_supported(const Dims& dm) {
+  return dm.dtype == LUKV_DTYPE_BF16 && dm.d == 128 && encode_fn() != nullptr;
+}
+
+cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const Workspace& ws, int32_t* dev_status,
+                            LaunchCtx& lc) {
+  CUtensorMap qm, km;
+  if (!make_map(&qm, q, (uint64_t)dm.heads() * dm.M) || !make_map(&km, k, (uint64_t)dm.heads() * dm.T))
+    return cudaErrorInvalidValue;
+  FusedArgs args;
+  args.stats = ws.stats;
+  args.lse = reinterpret_cast<float*>(reinterpret_cast<char*>(ws.head_flags) + lse_tag_offset(dm));
+  args.raw = ws.raw;
+  args.head_cnt = ws.head_flags;
+  args.dev_status = dev_status;
+  args.M = dm.M;
+  args.T = dm.T;
+  args.w = dm.w;
+  args.n = dm.n;
+  args.lse_rows = (dm.M + 1) & ~1;
+  args.head0 = 0;
+  args.nheads = (int)dm.heads();
+  args.item_tiles = score_item_tiles();
+  args.tiles_T = (dm.T + kTileKeys - 1) / kTileKeys;
+  args.tiles_n = (dm.n + kTileKeys - 1) / kTileKeys;
+  args.items_per_head = 0;  // set by the launcher
+  args.npad = (dm.M + 31) & ~31;
+  static const int hints = env_int("LUKV_L2_HINTS", 0, 1, 1);
+  args.l2_hints = hints;
+  static const int lag = env_int("LUKV_LAG", 2, kMaxLag, 3);
+  args.lag = lag;
+  args.scale_log2 = dm.scale_log2;
+  // the per-head counters and the (value, tag) rows must start at zero; they are adjacent in the workspace
+  cudaError_t e = cudaMemsetAsync(ws.head_flags, 0, score_tc_flag_bytes(dm), lc.st);
+  if (e != cudaSuccess) return e;
+  if (dm.M > 128) return launch_fused<2, 2>(qm, km, args, lc);
+  static const int quads = env_int("LUKV_QUADS", 2, 3, 2);
+  if (quads == 3) return launch_fused<1, 3>(qm, km, args, lc);
+  return launch_fused<1, 2>(qm, km, args, lc);
+}
+
+}  // namespace lukv
