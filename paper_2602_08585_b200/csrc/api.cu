@@ -94,12 +94,15 @@ static bool force_simt() {
   return v;
 }
 
+static HeadRange all_heads(const Dims& dm) { return HeadRange{0, (int)dm.heads()}; }
+
 static cudaError_t run_score(const Dims& dm, const void* q, const void* k, const Workspace& ws, float* pooled_out,
                              int32_t* dev_status, LaunchCtx& lc) {
-  cudaError_t e = (score_tc_supported(dm) && !force_simt()) ? launch_score_tc(dm, q, k, ws, dev_status, lc)
-                                                            : launch_score_simt(dm, q, k, ws, lc);
+  cudaError_t e = (score_tc_supported(dm) && !force_simt())
+                      ? launch_score_tc(dm, q, k, ws, dev_status, all_heads(dm), true, lc)
+                      : launch_score_simt(dm, q, k, ws, lc);
   if (e != cudaSuccess) return e;
-  return launch_pool(dm, ws.raw, pooled_out, lc);
+  return launch_pool(dm, ws.raw, pooled_out, all_heads(dm), lc);
 }
 
 // The whole path on one stream: allocation depends only on the curves, scoring only on Q/K;
@@ -110,8 +113,10 @@ static int run_compress(const Dims& dm, const void* q_win, const void* k, const 
   if (dev_status && cudaMemsetAsync(dev_status, 0, sizeof(int32_t), lc.st) != cudaSuccess) return LUKV_ERR_CUDA;
   if (launch_allocate(dm, curves, budgets_in, w.gains, budgets, offsets, lc) != cudaSuccess) return LUKV_ERR_CUDA;
   if (run_score(dm, q_win, k, w, w.pooled, dev_status, lc) != cudaSuccess) return LUKV_ERR_CUDA;
-  if (launch_select(dm, w.pooled, false, budgets, offsets, kept_idx, rows_cap, lc) != cudaSuccess) return LUKV_ERR_CUDA;
-  if (launch_gather(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (launch_select(dm, w.pooled, budgets, offsets, kept_idx, rows_cap, all_heads(dm), lc) != cudaSuccess)
+    return LUKV_ERR_CUDA;
+  if (launch_gather(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, all_heads(dm), lc) != cudaSuccess)
+    return LUKV_ERR_CUDA;
   return LUKV_OK;
 }
 
@@ -192,8 +197,10 @@ int lukv_select_gather(const lukv_params_t* params, const float* scores, const i
   if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;
-  if (launch_select(dm, scores, false, budgets, offsets, kept_idx, rows_cap, lc) != cudaSuccess) return LUKV_ERR_CUDA;
-  if (launch_gather(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (launch_select(dm, scores, budgets, offsets, kept_idx, rows_cap, all_heads(dm), lc) != cudaSuccess)
+    return LUKV_ERR_CUDA;
+  if (launch_gather(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, all_heads(dm), lc) != cudaSuccess)
+    return LUKV_ERR_CUDA;
   g_last_launches = lc.launches;
   return LUKV_OK;
 }

@@ -57,21 +57,26 @@ struct LaunchCtx {
   }
 };
 
+// Heads [h0, h0+nh) of the S*N heads of a call (the stages after allocation work head by head).
+struct HeadRange {
+  int h0, nh;
+};
+
 // Launchers.  Each returns cudaGetLastError() after its launches.
 cudaError_t launch_score_simt(const Dims& dm, const void* q, const void* k, const Workspace& ws, LaunchCtx& lc);
 // Folds per-chunk (max, sum-exp) partials [heads][chunks][M][2] into lse[heads][M] (exp2 domain).
 cudaError_t launch_lse(const Dims& dm, const float* stats, float* lse, int chunks, LaunchCtx& lc);
 // Tensor-core scorer (bf16, head_dim 128).  dev_status may be null.
 bool score_tc_supported(const Dims& dm);
+// clear_flags: zero the scorer's counters and (lse, tag) rows first (once per call, before the first range)
 cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const Workspace& ws, int32_t* dev_status,
-                            LaunchCtx& lc);
-cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, LaunchCtx& lc);
+                            HeadRange hr, bool clear_flags, LaunchCtx& lc);
+cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, HeadRange hr, LaunchCtx& lc);
 cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, float* gains,
                             int32_t* budgets, int32_t* offsets, LaunchCtx& lc);
-// scores_are_raw: apply the max-pool while loading (fused path) instead of expecting pooled input
-cudaError_t launch_select(const Dims& dm, const float* scores, bool scores_are_raw, const int32_t* budgets,
-                          const int32_t* offsets, int32_t* kept_idx, int64_t rows_cap, LaunchCtx& lc);
+cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* budgets, const int32_t* offsets,
+                          int32_t* kept_idx, int64_t rows_cap, HeadRange hr, LaunchCtx& lc);
 cudaError_t launch_gather(const Dims& dm, const int32_t* offsets, const int32_t* kept_idx, const void* k,
-                          const void* v, void* k_out, void* v_out, int64_t rows_cap, LaunchCtx& lc);
+                          const void* v, void* k_out, void* v_out, int64_t rows_cap, HeadRange hr, LaunchCtx& lc);
 
 }  // namespace lukv

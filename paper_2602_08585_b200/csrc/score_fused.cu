@@ -18,9 +18,9 @@
 // pass 2 needs it, and the key tiles pass 2 re-reads are still in L2: K crosses HBM once.
 //
 // Warp roles per CTA: 4*NQ epilogue warps in NQ quads (a warp may only read the TMEM lanes
-// 32*(warp%4)..+31), then one warp each: TMA producer, MMA issuer and TMEM owner, publisher
-// (pass-1 partials -> global memory, head completion), prefetcher (-lse -> shared memory).
-// The last two keep every global-memory round trip off the epilogue warps.
+// 32*(warp%4)..+31), then one warp each: TMA producer, MMA issuer 0 and TMEM owner, MMA issuer 1,
+// helper (pass-1 partials -> global memory, head completion, -lse -> shared memory: it keeps every
+// global-memory round trip off the epilogue warps).
 // Every wait is bounded; a wait that runs out raises the CTA's abort flag and stores
 // LUKV_ERR_TIMEOUT to the status word; the CTA then skips the remaining work and tears down
 // normally.
@@ -70,7 +70,8 @@ __device__ __forceinline__ void raise_abort(volatile int* abort_flag, int32_t* d
 }
 // Bounded wait: false when the CTA is aborting or the limit is reached (then it raises the abort).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
-  if (*abort_flag) return false;
+  // the common case (already complete) must not touch shared memory more than once: while the
+  // tensor pipe streams its operands, every shared-memory access costs ~100 cycles
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
@@ -230,11 +231,14 @@ template <int MT, int NQ>
 struct Plan {
   static_assert(MT == 1 || NQ == 2, "two query-row blocks are split over exactly two quads");
   static constexpr int kEpiWarps = 4 * NQ;
-  static constexpr int kThreads = (kEpiWarps + 4) * 32;  // + TMA producer, MMA issuer, publisher, prefetcher
-  static constexpr int kStages = MT == 1 ? 3 : 2;      // key-tile ring
+  // + TMA producer, two MMA issuers, helper.  The count stays a multiple of 4 warps: the register
+  // file is handed out as if the CTA were rounded up to one.
+  static constexpr int kThreads = (kEpiWarps + 4) * 32;
+  static constexpr int kStages = MT == 1 ? 4 : 2;      // key-tile ring: a stage is held from its TMA request until the
+                                                       // MMAs that read it complete, so HBM latency needs >= 4 of them
   static constexpr int kQSlots = 2;                    // query tiles of the job in the tensor pipe and the next one
   static constexpr int kQBytes = MT * kStageBytes;     // [half][MT*128 rows][128 B]
-  static constexpr int kFinBufs = MT == 1 ? 2 : 1;     // blocks of partials in flight while a head is folded
+  static constexpr int kFinBufs = 1;                   // blocks of partials in flight while a head is folded
   static constexpr int kFinParts = kFinBytes / (128 * MT * 8);  // partials per block
   static constexpr int kKOff = kQSlots * kQBytes;
   static constexpr int kFinOff = kKOff + kStages * kStageBytes;
@@ -385,7 +389,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
     }
     for (int s = 0; s < P::kQSlots; ++s) {
       mbar_init(bar(P::kBarQFull, s), 1);
-      mbar_init(bar(P::kBarQEmpty, s), 1);
+      mbar_init(bar(P::kBarQEmpty, s), 2);  // both MMA issuers
     }
     for (int b = 0; b < kNumBufs; ++b) {
       mbar_init(bar(P::kBarTFull, b), 1);
@@ -447,18 +451,27 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
         if (!ok) break;
       }
     }
-  } else if (warp == kEpiWarps + 1) {
-    // ---------------- MMA issuer ----------------
+  } else if (warp == kEpiWarps + 1 || warp == kEpiWarps + 2) {
+    // ---------------- MMA issuers ----------------
+    // Two threads (in two warps) issue alternate key tiles.  A thread is held up by its waits and by
+    // the tensor pipe's issue queue; with two of them one can wait while the other issues, so the
+    // pipe does not idle between tiles.  Tiles that share an accumulator buffer or a key stage
+    // (both have an even count) always belong to the same issuer, which keeps them in order.
     if (lane == 0) {
+      const uint32_t me = warp == kEpiWarps + 1 ? 0u : 1u;
       uint32_t tt = 0, jq = 0;
       for (int idx = 0; idx < njobs; ++idx) {
         const Job j = decode_job(idx, K, a);
         if (j.ntiles == 0) continue;
         const uint32_t slot = jq % P::kQSlots;
-        if (!mbar_wait(bar(P::kBarQFull, slot), (jq / P::kQSlots) & 1, abort_flag, a.dev_status)) break;
         const uint32_t qd = q_s + slot * P::kQBytes;
-        bool ok = true;
+        bool ok = true, have_q = false;
         for (int t = 0; t < j.ntiles; ++t, ++tt) {
+          if ((tt & 1) != me) continue;
+          if (!have_q) {
+            if (!(ok = mbar_wait(bar(P::kBarQFull, slot), (jq / P::kQSlots) & 1, abort_flag, a.dev_status))) break;
+            have_q = true;
+          }
           const uint32_t s = tt % kStages, ph = (tt / kStages) & 1;
           const uint32_t buf = tt % kNumBufs, use = tt / kNumBufs;
           if (!(ok = mbar_wait(bar(P::kBarTEmpty, buf), (use & 1) ^ 1, abort_flag, a.dev_status))) break;
@@ -493,150 +506,171 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
           umma_commit(bar(P::kBarTFull, buf));   // the accumulator is complete
         }
         if (!ok) break;
-        umma_commit(bar(P::kBarQEmpty, slot));   // the query tiles may be replaced
+        umma_commit(bar(P::kBarQEmpty, slot));   // this issuer's share of the job no longer needs the query tiles
         ++jq;
       }
     }
-  } else if (warp == kEpiWarps + 2) {
-    // ---------------- publisher: pass-1 partials -> global memory, head completion ----------------
-    // For item k: merge the quads' partials, store them, count the item in (release).  The warp
-    // that counts a head's last item folds all its partials into the row log-sum-exp and stores
-    // it as (value, tag) pairs, which the prefetchers of the head's CTAs poll.
+  } else if (warp == kEpiWarps + 3) {
+    // ---------------- helper: everything that needs a global-memory round trip ----------------
+    // publish(k): merge the quads' pass-1 partials of item k, store them, count the item in
+    //   (release).  The warp that counts a head's last item folds all its partials into the row
+    //   log-sum-exp and stores it as (value, tag) pairs, zero at launch.
+    // prefetch(k): poll those pairs for the head of item k (polling the data itself saves a flag
+    //   round trip) and put -lse into shared memory for pass 2 of item k, which the quads reach
+    //   several jobs after its pass 1.
+    // Both are attempted in turn without blocking, so a head that completes late does not hold up
+    // the publication of this CTA's next partials.
     uint32_t fin_uses[P::kFinBufs] = {};
-    for (int k = 0; k < K; ++k) {
-      const Job j1 = make_job(k, false, a);
-      bool ok = true;
-      for (int q = 0; q < NQ; ++q) ok = mbar_wait(bar(P::kBarPubFull, q), k & 1, abort_flag, a.dev_status) && ok;
-      if (ok) {
-        float2* dst = reinterpret_cast<float2*>(a.stats) + ((size_t)j1.u * a.items_per_head + j1.c) * kRowsPad;
-#pragma unroll
-        for (int rr = 0; rr < kRowsPad; rr += 32) {
-          float2 v = pub_s[rr + lane];
-          if (MT == 1) {
-            // the quads hold partials of the same 128 rows over different key tiles: merge them
-#pragma unroll
-            for (int q = 1; q < NQ; ++q) {
-              const float2 o = pub_s[q * 128 + rr + lane];
-              if (o.y > 0.f) {  // an empty partial is (-inf, 0)
-                const float mn = fmaxf(v.x, o.x);
-                v.y = v.y * ex2(v.x - mn) + o.y * ex2(o.x - mn);
-                v.x = mn;
-              }
-            }
-          }
-          dst[rr + lane] = v;  // rows beyond M carry (-inf, 0)
-        }
-      }
-      __syncwarp();
-      if (lane == 0 && ok)
-        for (int q = 0; q < NQ; ++q) mbar_arrive(bar(P::kBarPubEmpty, q), 1);
-      // count the item in (release: the partials above; acquire: everybody else's)
-      int last = 0;
-      if (lane == 0 && ok && !*abort_flag) last = atom_add_acq_rel(a.head_cnt + j1.u, 1) == a.items_per_head - 1;
-      last = __shfl_sync(0xffffffffu, last, 0);
-      if (last) {
-        // Fold the head's partials: the bulk-copy engine brings them into shared memory in blocks of
-        // kFinParts items (one round trip per block instead of one per load); every lane folds its rows.
-        constexpr int kRowsLane = 4 * MT;
-        const char* src = reinterpret_cast<const char*>(a.stats) + (size_t)j1.u * a.items_per_head * kRowsPad * 8;
-        const int nblk = (a.items_per_head + P::kFinParts - 1) / P::kFinParts;
-        auto request = [&](int blk) {  // lane 0
-          const int parts = min(P::kFinParts, a.items_per_head - blk * P::kFinParts);
-          const uint32_t bytes = (uint32_t)parts * kRowsPad * 8, b = blk % P::kFinBufs;
-          mbar_expect_tx(bar(P::kBarFin, b), bytes);
-          bulk_load(sbase + P::kFinOff + b * kFinBytes, src + (size_t)blk * P::kFinParts * kRowsPad * 8, bytes,
-                    bar(P::kBarFin, b));
-        };
-        asm volatile("fence.proxy.async;" ::: "memory");
+    constexpr int kRowsLaneP = 4 * MT;
+    int kp = 0, kf = 0;
+    uint32_t p2c = 0, idle = 0;
+    while ((kp < K || kf < K) && !*abort_flag) {
+      bool progress = false;
+      if (kp < K) {
+        int ready = 1;
         if (lane == 0)
-          for (int blk = 0; blk < nblk && blk < P::kFinBufs; ++blk) request(blk);
-        float fm[kRowsLane], fl[kRowsLane];
+          for (int q = 0; q < NQ; ++q) ready &= (int)mbar_try_wait(bar(P::kBarPubFull, q), kp & 1);
+        ready = __shfl_sync(0xffffffffu, ready, 0);
+        if (ready) {
+          const int k = kp;
+          const bool ok = true;
+          const Job j1 = make_job(k, false, a);
+          if (ok) {
+            float2* dst = reinterpret_cast<float2*>(a.stats) + ((size_t)j1.u * a.items_per_head + j1.c) * kRowsPad;
 #pragma unroll
-        for (int jj = 0; jj < kRowsLane; ++jj) fm[jj] = -INFINITY, fl[jj] = 0.f;
-        bool fin_ok = true;
-        for (int blk = 0; blk < nblk; ++blk) {
-          const uint32_t b = blk % P::kFinBufs;
-          fin_ok = fin_ok && mbar_wait(bar(P::kBarFin, b), fin_uses[b] & 1, abort_flag, a.dev_status);
-          ++fin_uses[b];
-          if (fin_ok) {
-            const float2* part = reinterpret_cast<const float2*>(smem + P::kFinOff + b * kFinBytes);
-            const int parts = min(P::kFinParts, a.items_per_head - blk * P::kFinParts);
-            float cm[kRowsLane], cl[kRowsLane];
+            for (int rr = 0; rr < kRowsPad; rr += 32) {
+              float2 v = pub_s[rr + lane];
+              if (MT == 1) {
+                // the quads hold partials of the same 128 rows over different key tiles: merge them
 #pragma unroll
-            for (int jj = 0; jj < kRowsLane; ++jj) cm[jj] = fm[jj], cl[jj] = 0.f;
-            for (int c = 0; c < parts; ++c)
-#pragma unroll
-              for (int jj = 0; jj < kRowsLane; ++jj) {
-                const float2 v = part[c * kRowsPad + 32 * jj + lane];
-                if (v.y > 0.f) cm[jj] = fmaxf(cm[jj], v.x);  // an empty partial is (-inf, 0)
+                for (int q = 1; q < NQ; ++q) {
+                  const float2 o = pub_s[q * 128 + rr + lane];
+                  if (o.y > 0.f) {  // an empty partial is (-inf, 0)
+                    const float mn = fmaxf(v.x, o.x);
+                    v.y = v.y * ex2(v.x - mn) + o.y * ex2(o.x - mn);
+                    v.x = mn;
+                  }
+                }
               }
-            for (int c = 0; c < parts; ++c)
-#pragma unroll
-              for (int jj = 0; jj < kRowsLane; ++jj) {
-                const float2 v = part[c * kRowsPad + 32 * jj + lane];
-                if (v.y > 0.f) cl[jj] = fmaf(v.y, ex2(v.x - cm[jj]), cl[jj]);
-              }
-#pragma unroll
-            for (int jj = 0; jj < kRowsLane; ++jj)
-              if (cl[jj] > 0.f) {
-                fl[jj] = fmaf(fl[jj], ex2(fm[jj] - cm[jj]), cl[jj]);
-                fm[jj] = cm[jj];
-              }
+              dst[rr + lane] = v;  // rows beyond M carry (-inf, 0)
+            }
           }
           __syncwarp();
-          if (lane == 0 && fin_ok && blk + P::kFinBufs < nblk) request(blk + P::kFinBufs);
-        }
-        float2* out = reinterpret_cast<float2*>(a.lse) + (size_t)j1.u * a.lse_rows;
+          if (lane == 0 && ok)
+            for (int q = 0; q < NQ; ++q) mbar_arrive(bar(P::kBarPubEmpty, q), 1);
+          // count the item in (release: the partials above; acquire: everybody else's)
+          int last = 0;
+          if (lane == 0 && ok && !*abort_flag) last = atom_add_acq_rel(a.head_cnt + j1.u, 1) == a.items_per_head - 1;
+          last = __shfl_sync(0xffffffffu, last, 0);
+          if (last) {
+            // Fold the head's partials: the bulk-copy engine brings them into shared memory in blocks of
+            // kFinParts items (one round trip per block instead of one per load); every lane folds its rows.
+            constexpr int kRowsLane = 4 * MT;
+            const char* src = reinterpret_cast<const char*>(a.stats) + (size_t)j1.u * a.items_per_head * kRowsPad * 8;
+            const int nblk = (a.items_per_head + P::kFinParts - 1) / P::kFinParts;
+            auto request = [&](int blk) {  // lane 0
+              const int parts = min(P::kFinParts, a.items_per_head - blk * P::kFinParts);
+              const uint32_t bytes = (uint32_t)parts * kRowsPad * 8, b = blk % P::kFinBufs;
+              mbar_expect_tx(bar(P::kBarFin, b), bytes);
+              bulk_load(sbase + P::kFinOff + b * kFinBytes, src + (size_t)blk * P::kFinParts * kRowsPad * 8, bytes,
+                        bar(P::kBarFin, b));
+            };
+            asm volatile("fence.proxy.async;" ::: "memory");
+            if (lane == 0)
+              for (int blk = 0; blk < nblk && blk < P::kFinBufs; ++blk) request(blk);
+            float fm[kRowsLane], fl[kRowsLane];
 #pragma unroll
-        for (int jj = 0; jj < kRowsLane; ++jj) {
-          const int row = 32 * jj + lane;
-          if (row < a.lse_rows && fin_ok) __stcg(out + row, make_float2(fm[jj] + log2f(fl[jj]), 1.f));
-        }
-      }
-    }
-  } else if (warp == kEpiWarps + 3) {
-    // ---------------- prefetcher: -lse of the pass-2 jobs to come -> shared memory ----------------
-    // The log-sum-exp rows are stored as (value, tag) pairs that are zero at launch; polling the
-    // data itself saves a flag round trip.  The quads reach pass 2 of item k several jobs after its
-    // pass 1, so this latency is normally hidden.
-    constexpr int kRowsLane = 4 * MT;
-    uint32_t p2c = 0;
-    for (int k = 0; k < K; ++k) {
-      const Job j2 = make_job(k, true, a);
-      if (j2.ntiles == 0) continue;
-      const uint32_t slot = p2c % a.lag;
-      const bool ok = mbar_wait(bar(P::kBarLseEmpty, slot), ((p2c / a.lag) & 1) ^ 1, abort_flag, a.dev_status);
-      const float2* src = reinterpret_cast<const float2*>(a.lse) + (size_t)j2.u * a.lse_rows;
-      float2 v[kRowsLane];
-      bool have = false;
-      if (ok) {
-        for (uint32_t spin = 0; spin < kSpinLimit && !have; ++spin) {
-          bool mine = true;
+            for (int jj = 0; jj < kRowsLane; ++jj) fm[jj] = -INFINITY, fl[jj] = 0.f;
+            bool fin_ok = true;
+            for (int blk = 0; blk < nblk; ++blk) {
+              const uint32_t b = blk % P::kFinBufs;
+              fin_ok = fin_ok && mbar_wait(bar(P::kBarFin, b), fin_uses[b] & 1, abort_flag, a.dev_status);
+              ++fin_uses[b];
+              if (fin_ok) {
+                const float2* part = reinterpret_cast<const float2*>(smem + P::kFinOff + b * kFinBytes);
+                const int parts = min(P::kFinParts, a.items_per_head - blk * P::kFinParts);
+                float cm[kRowsLane], cl[kRowsLane];
 #pragma unroll
-          for (int jj = 0; jj < kRowsLane; ++jj) {
-            const int row = 32 * jj + lane;
-            if (row < a.M) {
-              v[jj] = ld_relaxed_f2(src + row);
-              mine = mine && v[jj].y != 0.f;
+                for (int jj = 0; jj < kRowsLane; ++jj) cm[jj] = fm[jj], cl[jj] = 0.f;
+                for (int c = 0; c < parts; ++c)
+#pragma unroll
+                  for (int jj = 0; jj < kRowsLane; ++jj) {
+                    const float2 v = part[c * kRowsPad + 32 * jj + lane];
+                    if (v.y > 0.f) cm[jj] = fmaxf(cm[jj], v.x);  // an empty partial is (-inf, 0)
+                  }
+                for (int c = 0; c < parts; ++c)
+#pragma unroll
+                  for (int jj = 0; jj < kRowsLane; ++jj) {
+                    const float2 v = part[c * kRowsPad + 32 * jj + lane];
+                    if (v.y > 0.f) cl[jj] = fmaf(v.y, ex2(v.x - cm[jj]), cl[jj]);
+                  }
+#pragma unroll
+                for (int jj = 0; jj < kRowsLane; ++jj)
+                  if (cl[jj] > 0.f) {
+                    fl[jj] = fmaf(fl[jj], ex2(fm[jj] - cm[jj]), cl[jj]);
+                    fm[jj] = cm[jj];
+                  }
+              }
+              __syncwarp();
+              if (lane == 0 && fin_ok && blk + P::kFinBufs < nblk) request(blk + P::kFinBufs);
+            }
+            float2* out = reinterpret_cast<float2*>(a.lse) + (size_t)j1.u * a.lse_rows;
+#pragma unroll
+            for (int jj = 0; jj < kRowsLane; ++jj) {
+              const int row = 32 * jj + lane;
+              if (row < a.lse_rows && fin_ok) __stcg(out + row, make_float2(fm[jj] + log2f(fl[jj]), 1.f));
             }
           }
-          have = __all_sync(0xffffffffu, mine);
-          if (!have) {
-            if (*abort_flag) break;
-            if (spin > 16) __nanosleep(200);
+          ++kp;
+          progress = true;
+        }
+      }
+      if (kf < kp) {
+        const Job j2 = make_job(kf, true, a);
+        if (j2.ntiles == 0) {
+          ++kf;
+          progress = true;
+        } else {
+          const uint32_t slot = p2c % a.lag;
+          int freeslot = 0;
+          if (lane == 0) freeslot = (int)mbar_try_wait(bar(P::kBarLseEmpty, slot), ((p2c / a.lag) & 1) ^ 1);
+          freeslot = __shfl_sync(0xffffffffu, freeslot, 0);
+          if (freeslot) {
+            const float2* src = reinterpret_cast<const float2*>(a.lse) + (size_t)j2.u * a.lse_rows;
+            float2 v[kRowsLaneP];
+            bool mine = true;
+#pragma unroll
+            for (int jj = 0; jj < kRowsLaneP; ++jj) {
+              const int row = 32 * jj + lane;
+              if (row < a.M) {
+                v[jj] = ld_relaxed_f2(src + row);
+                mine = mine && v[jj].y != 0.f;
+              }
+            }
+            if (__all_sync(0xffffffffu, mine)) {
+#pragma unroll
+              for (int jj = 0; jj < 8; ++jj) {
+                const int row = 32 * jj + lane;
+                nlse_s[slot * 256 + row] = (jj < kRowsLaneP && row < a.M) ? -v[jj < kRowsLaneP ? jj : 0].x : -INFINITY;
+              }
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bar(P::kBarLseFull, slot), 1);
+              ++p2c;
+              ++kf;
+              progress = true;
+            }
           }
         }
-        if (!have && lane == 0 && !*abort_flag) raise_abort(abort_flag, a.dev_status);
       }
-      __syncwarp();
-#pragma unroll
-      for (int jj = 0; jj < 8; ++jj) {
-        const int row = 32 * jj + lane;
-        nlse_s[slot * 256 + row] = (have && jj < kRowsLane && row < a.M) ? -v[jj < kRowsLane ? jj : 0].x : -INFINITY;
+      if (progress) {
+        idle = 0;
+      } else {
+        if (++idle > kSpinLimit) {
+          if (lane == 0) raise_abort(abort_flag, a.dev_status);
+          break;
+        }
+        if (idle > 8) __nanosleep(100);
       }
-      __syncwarp();
-      if (lane == 0 && ok) mbar_arrive(bar(P::kBarLseFull, slot), 1);
-      ++p2c;
     }
   } else {
     // ---------------- epilogue quads ----------------
@@ -834,7 +868,7 @@ bool score_tc_supported(const Dims& dm) {
 }
 
 cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const Workspace& ws, int32_t* dev_status,
-                            LaunchCtx& lc) {
+                            HeadRange hr, bool clear_flags, LaunchCtx& lc) {
   CUtensorMap qm, km;
   if (!make_map(&qm, q, (uint64_t)dm.heads() * dm.M) || !make_map(&km, k, (uint64_t)dm.heads() * dm.T))
     return cudaErrorInvalidValue;
@@ -849,8 +883,8 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
   args.w = dm.w;
   args.n = dm.n;
   args.lse_rows = (dm.M + 1) & ~1;
-  args.head0 = 0;
-  args.nheads = (int)dm.heads();
+  args.head0 = hr.h0;
+  args.nheads = hr.nh;
   args.item_tiles = score_item_tiles();
   args.tiles_T = (dm.T + kTileKeys - 1) / kTileKeys;
   args.tiles_n = (dm.n + kTileKeys - 1) / kTileKeys;
@@ -862,8 +896,10 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
   args.lag = lag;
   args.scale_log2 = dm.scale_log2;
   // the per-head counters and the (value, tag) rows must start at zero; they are adjacent in the workspace
-  cudaError_t e = cudaMemsetAsync(ws.head_flags, 0, score_tc_flag_bytes(dm), lc.st);
-  if (e != cudaSuccess) return e;
+  if (clear_flags) {
+    const cudaError_t e = cudaMemsetAsync(ws.head_flags, 0, score_tc_flag_bytes(dm), lc.st);
+    if (e != cudaSuccess) return e;
+  }
   if (dm.M > 128) return launch_fused<2, 2>(qm, km, args, lc);
   static const int quads = env_int("LUKV_QUADS", 2, 3, 2);
   if (quads == 3) return launch_fused<1, 3>(qm, km, args, lc);

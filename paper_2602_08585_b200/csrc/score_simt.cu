@@ -198,8 +198,8 @@ __global__ void score_lse_kernel(const float* __restrict__ stats, float* __restr
 }
 
 __global__ void max_pool_kernel(const float* __restrict__ raw, float* __restrict__ pooled, int n, int half,
-                                int tiles) {
-  const int u = blockIdx.x / tiles;
+                                int tiles, int head0) {
+  const int u = head0 + blockIdx.x / tiles;
   const int j = (blockIdx.x % tiles) * blockDim.x + threadIdx.x;
   if (j >= n) return;
   const float* r = raw + (size_t)u * n;
@@ -260,9 +260,9 @@ cudaError_t launch_lse(const Dims& dm, const float* stats, float* lse, int chunk
   return cudaGetLastError();
 }
 
-cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, LaunchCtx& lc) {
+cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, HeadRange hr, LaunchCtx& lc) {
   const int tiles = (dm.n + 255) / 256;
-  max_pool_kernel<<<(unsigned)(dm.heads() * tiles), 256, 0, lc.st>>>(raw, pooled, dm.n, dm.kp / 2, tiles);
+  max_pool_kernel<<<(unsigned)((int64_t)hr.nh * tiles), 256, 0, lc.st>>>(raw, pooled, dm.n, dm.kp / 2, tiles, hr.h0);
   lc.mark("max_pool");
   return cudaGetLastError();
 }

@@ -45,10 +45,10 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
                                                                 const int32_t* __restrict__ budgets,
                                                                 const int32_t* __restrict__ offsets,
                                                                 int32_t* __restrict__ kept_idx, long long rows_cap,
-                                                                int n, int w, int span_rt) {
+                                                                int n, int w, int span_rt, int head0) {
   __shared__ __align__(16) int cnt_buf[2][kSelWarps];
   __shared__ int scan_gt[kSelWarps], scan_eq[kSelWarps];
-  const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
+  const int u = head0 + blockIdx.x, tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
   const int b = budgets[u];
   const long long off = offsets[u];
   const float* src = pooled + (size_t)u * n;
@@ -162,9 +162,10 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(const int32_t* _
                                                                 const int32_t* __restrict__ kept_idx,
                                                                 const uint4* __restrict__ k, const uint4* __restrict__ v,
                                                                 uint4* __restrict__ k_out, uint4* __restrict__ v_out,
-                                                                long long rows_cap, int heads, int T) {
-  // rows actually present: the last offset, clipped to what the output can hold
-  const long long total_rows = min((long long)__ldg(offsets + heads), rows_cap);
+                                                                long long rows_cap, int head0, int nheads, int T) {
+  // packed rows of heads [head0, head0+nheads), clipped to what the output can hold
+  const long long row_begin = __ldg(offsets + head0);
+  const long long total_rows = min((long long)__ldg(offsets + head0 + nheads), rows_cap);
   constexpr int kRowsPerBatch = 32 / LPR;
   constexpr int kBatches = 32 / kRowsPerBatch;  // == LPR
   constexpr int kInFlight = LPR < 4 ? LPR : 4;
@@ -172,11 +173,11 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(const int32_t* _
   const long long warp_global = ((long long)blockIdx.x * kGatherThreads + threadIdx.x) >> 5;
   const long long warps_total = ((long long)gridDim.x * kGatherThreads) >> 5;
   const int sub = lane / LPR, part = lane % LPR;
-  for (long long base = warp_global * 32; base < total_rows; base += warps_total * 32) {
+  for (long long base = row_begin + warp_global * 32; base < total_rows; base += warps_total * 32) {
     const long long r = base + lane;
     long long src_row = -1;
     if (r < total_rows) {
-      int lo = 0, hi = heads;  // largest u with offsets[u] <= r
+      int lo = head0, hi = head0 + nheads;  // largest u with offsets[u] <= r
       while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
         if ((long long)__ldg(offsets + mid) <= r) lo = mid; else hi = mid;
@@ -210,49 +211,49 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(const int32_t* _
 
 template <int LPR>
 void launch_gather_t(const Dims& dm, const int32_t* offsets, const int32_t* kept_idx, const void* k, const void* v,
-                     void* k_out, void* v_out, long long rows_cap, cudaStream_t st) {
-  const long long spans = (rows_cap + 31) / 32;
+                     void* k_out, void* v_out, long long rows_cap, HeadRange hr, cudaStream_t st) {
+  // the rows of a head range are only known on the device; size the grid for its share of the output
+  const long long spans = (rows_cap * hr.nh / (long long)dm.heads() + 31) / 32 + 1;
   long long blocks = (spans + kGatherThreads / 32 - 1) / (kGatherThreads / 32);
   const long long max_blocks = 148LL * 8 * 4;  // a few waves of resident CTAs; the loop covers the rest
   if (blocks > max_blocks) blocks = max_blocks;
   if (blocks < 1) blocks = 1;
   gather_kernel<LPR><<<(unsigned)blocks, kGatherThreads, 0, st>>>(offsets, kept_idx, (const uint4*)k, (const uint4*)v,
-                                                                  (uint4*)k_out, (uint4*)v_out, rows_cap,
-                                                                  (int)dm.heads(), dm.T);
+                                                                  (uint4*)k_out, (uint4*)v_out, rows_cap, hr.h0,
+                                                                  hr.nh, dm.T);
 }
 
 }  // namespace
 
-cudaError_t launch_select(const Dims& dm, const float* scores, bool scores_are_raw, const int32_t* budgets,
-                          const int32_t* offsets, int32_t* kept_idx, int64_t rows_cap, LaunchCtx& lc) {
+cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* budgets, const int32_t* offsets,
+                          int32_t* kept_idx, int64_t rows_cap, HeadRange hr, LaunchCtx& lc) {
   cudaStream_t st = lc.st;
-  (void)scores_are_raw;  // pooling is done by launch_pool before this call
-  const unsigned grid = (unsigned)dm.heads();
+  const unsigned grid = (unsigned)hr.nh;
   const int n = dm.n;
   if (n <= kSelThreads * 4)
-    select_kernel<4><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0);
+    select_kernel<4><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0);
   else if (n <= kSelThreads * 16)
-    select_kernel<16><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0);
+    select_kernel<16><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0);
   else if (n <= kSelThreads * 64)
-    select_kernel<64><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0);
+    select_kernel<64><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0);
   else {
     const int per_warp = (n + kSelWarps - 1) / kSelWarps;
     const int span = (per_warp + 31) & ~31;
-    select_kernel<0><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, span);
+    select_kernel<0><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, span, hr.h0);
   }
   lc.mark("select");
   return cudaGetLastError();
 }
 
 cudaError_t launch_gather(const Dims& dm, const int32_t* offsets, const int32_t* kept_idx, const void* k,
-                          const void* v, void* k_out, void* v_out, int64_t rows_cap, LaunchCtx& lc) {
+                          const void* v, void* k_out, void* v_out, int64_t rows_cap, HeadRange hr, LaunchCtx& lc) {
   cudaStream_t st = lc.st;
   if (rows_cap <= 0) return cudaSuccess;
   const int lpr = (int)(dm.d * dm.esize() / 16);
   switch (lpr) {
-    case 8: launch_gather_t<8>(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, st); break;
-    case 16: launch_gather_t<16>(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, st); break;
-    default: launch_gather_t<32>(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, st); break;
+    case 8: launch_gather_t<8>(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, hr, st); break;
+    case 16: launch_gather_t<16>(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, hr, st); break;
+    default: launch_gather_t<32>(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, hr, st); break;
   }
   lc.mark("gather");
   return cudaGetLastError();
