@@ -13,11 +13,20 @@ namespace {
 
 // ---- hull ----------------------------------------------------------------------------
 
-// mean(a/b) <= mean(c/d) decided exactly as the comparison of the two correctly rounded
-// fp64 quotients (b, d > 0).  The products decide whenever they are clearly apart (then the
-// rounded quotients are ordered the same way); otherwise the quotients themselves are
-// compared.
-__device__ __forceinline__ bool mean_le(double a, double b, double c, double d) {
+// mean of block [l1,r1) <= mean of block [l2,r2), where the mean of [l,r) is (U[r]-U[l])/(r-l),
+// decided exactly as the comparison of the two correctly rounded fp64 quotients.  Three tiers,
+// cheapest first (the fp64 pipe is slow, and the walk below is one dependent chain):
+//   fp32 cross products, when they are further apart than fp32 rounding can explain;
+//   fp64 cross products, when they are clearly apart;
+//   the fp64 quotients themselves.
+__device__ __forceinline__ bool mean_le(const float* U, int l1, int r1, int l2, int r2) {
+  const float fa = U[r1] - U[l1], fb = (float)(r1 - l1), fc = U[r2] - U[l2], fd = (float)(r2 - l2);
+  const float q1 = fa * fd, q2 = fc * fb;
+  const float ftol = 4e-7f * fmaxf(fabsf(q1), fabsf(q2));  // each product carries two roundings of 2^-24
+  if (q1 < q2 - ftol) return true;
+  if (q1 > q2 + ftol) return false;
+  const double a = __dsub_rn((double)U[r1], (double)U[l1]), b = (double)(r1 - l1);
+  const double c = __dsub_rn((double)U[r2], (double)U[l2]), d = (double)(r2 - l2);
   const double p1 = __dmul_rn(a, d), p2 = __dmul_rn(c, b);
   const double diff = __dsub_rn(p1, p2);
   const double tol = fmax(fabs(p1), fabs(p2)) * 9.094947017729282e-13;  // 2^-40
@@ -25,6 +34,9 @@ __device__ __forceinline__ bool mean_le(double a, double b, double c, double d) 
   if (diff > tol) return false;
   return __ddiv_rn(a, b) <= __ddiv_rn(c, d);
 }
+
+// Shared memory of one warp of the hull kernel: [P] floats, [P] ints, [P] floats.
+__host__ __device__ inline size_t hull_bytes_per_warp(int P) { return ((size_t)P * 12 + 15) & ~(size_t)15; }
 
 // One warp per head.  Lane 0 runs the pool-adjacent-violators stack (the sequence of merge
 // decisions is the algorithm; it is serial by nature) with the top block cached in registers;
@@ -36,35 +48,23 @@ __global__ void hull_kernel(const float* __restrict__ curves, float* __restrict_
   const int warps = blockDim.x >> 5;
   const int hid = blockIdx.x * warps + warp;
   if (hid >= N) return;  // whole warps leave together; only __syncwarp is used below
-  float* Us = reinterpret_cast<float*>(hull_smem) + (size_t)warp * 3 * P;  // [P] curve
-  int* Ls = reinterpret_cast<int*>(Us + P);                                // [P] stack of block starts
-  float* Gs = Us + 2 * P;                                                   // [P-1] gains
+  float* Us = reinterpret_cast<float*>(hull_smem + (size_t)warp * hull_bytes_per_warp(P));  // [P] curve
+  int* Ls = reinterpret_cast<int*>(Us + P);                                                  // [P] stack of block starts
+  float* Gs = Us + 2 * P;                                                                     // [P-1] gains
   for (int p = lane; p < P; p += 32) Us[p] = curves[(size_t)hid * P + p];
   __syncwarp();
   int sp = 0;
   if (lane == 0) {
-    int top_l = 0;
-    double top_num = 0.0, top_den = 1.0;
+    int top_l = 0;  // start of the block on top of the stack; it ends where the current block starts
     for (int k = 0; k + 1 < P; ++k) {
       int cur_l = k;
-      const double u_r = (double)Us[k + 1];
-      double cur_num = __dsub_rn(u_r, (double)Us[k]);
-      double cur_den = 1.0;
-      while (sp > 0 && mean_le(top_num, top_den, cur_num, cur_den)) {
+      while (sp > 0 && mean_le(Us, top_l, cur_l, cur_l, k + 1)) {
         cur_l = top_l;
         --sp;
-        cur_num = __dsub_rn(u_r, (double)Us[cur_l]);
-        cur_den = (double)(k + 1 - cur_l);
-        if (sp > 0) {
-          top_l = Ls[sp - 1];
-          top_num = __dsub_rn((double)Us[cur_l], (double)Us[top_l]);
-          top_den = (double)(cur_l - top_l);
-        }
+        if (sp > 0) top_l = Ls[sp - 1];
       }
       Ls[sp++] = cur_l;
       top_l = cur_l;
-      top_num = cur_num;
-      top_den = cur_den;
     }
   }
   sp = __shfl_sync(0xffffffffu, sp, 0);
@@ -283,10 +283,10 @@ __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __r
 cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, float* gains,
                             int32_t* budgets, int32_t* offsets, LaunchCtx& lc) {
   cudaStream_t st = lc.st;
-  // hull: one warp per head, up to 4 warps per block (3 arrays of P words per warp)
-  int hw = (int)((200u * 1024u) / ((size_t)dm.P * 12u));
+  // hull: one warp per head, up to 4 warps per block (12 bytes of shared memory per curve point and warp)
+  int hw = (int)((200u * 1024u) / hull_bytes_per_warp(dm.P));
   hw = hw > 4 ? 4 : (hw < 1 ? 1 : hw);
-  const size_t hull_smem = (size_t)dm.P * hw * 12;
+  const size_t hull_smem = hull_bytes_per_warp(dm.P) * hw;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(hull_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hull_smem)) != cudaSuccess)
     return e;

@@ -99,20 +99,66 @@ static HeadRange all_heads(const Dims& dm) { return HeadRange{0, (int)dm.heads()
 static cudaError_t run_score(const Dims& dm, const void* q, const void* k, const Workspace& ws, float* pooled_out,
                              int32_t* dev_status, LaunchCtx& lc) {
   cudaError_t e = (score_tc_supported(dm) && !force_simt())
-                      ? launch_score_tc(dm, q, k, ws, dev_status, all_heads(dm), true, lc)
+                      ? launch_score_tc(dm, q, k, ws, dev_status, all_heads(dm), true, 0, lc)
                       : launch_score_simt(dm, q, k, ws, lc);
   if (e != cudaSuccess) return e;
   return launch_pool(dm, ws.raw, pooled_out, all_heads(dm), lc);
 }
 
-// The whole path on one stream: allocation depends only on the curves, scoring only on Q/K;
-// selection needs both, the gather follows.
+// An auxiliary stream and the two events that tie it to the caller's stream, created on first
+// use on a device and kept until the process exits (handles only, no device memory).
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  bool ok = false;
+};
+static SideStream* side_stream() {
+  static SideStream table[64];
+  static std::mutex mu;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  SideStream& s = table[dev];
+  if (!s.ok) {
+    if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess)
+      return nullptr;
+    s.ok = true;
+  }
+  return &s;
+}
+
+// The whole path.  Allocation depends only on the curves, scoring only on Q/K; selection needs
+// both, the gather follows.  With `overlap` the two allocation kernels run on an auxiliary stream
+// beside the scorer, which then leaves two SMs to them (its CTAs fill theirs completely); the
+// caller's stream waits for the budgets before selection, so stream order is preserved.
 static int run_compress(const Dims& dm, const void* q_win, const void* k, const void* v, const float* curves,
                         const int64_t* budgets_in, void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets,
-                        int32_t* offsets, int64_t rows_cap, int32_t* dev_status, const Workspace& w, LaunchCtx& lc) {
+                        int32_t* offsets, int64_t rows_cap, int32_t* dev_status, const Workspace& w, LaunchCtx& lc,
+                        bool overlap) {
   if (dev_status && cudaMemsetAsync(dev_status, 0, sizeof(int32_t), lc.st) != cudaSuccess) return LUKV_ERR_CUDA;
-  if (launch_allocate(dm, curves, budgets_in, w.gains, budgets, offsets, lc) != cudaSuccess) return LUKV_ERR_CUDA;
-  if (run_score(dm, q_win, k, w, w.pooled, dev_status, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  const bool tc = score_tc_supported(dm) && !force_simt();
+  SideStream* side = (overlap && tc) ? side_stream() : nullptr;
+  int rc = LUKV_OK;
+  if (side) {
+    LaunchCtx ls;
+    ls.st = side->stream;
+    if (cudaEventRecord(side->fork, lc.st) != cudaSuccess || cudaStreamWaitEvent(ls.st, side->fork, 0) != cudaSuccess)
+      return LUKV_ERR_CUDA;
+    if (launch_allocate(dm, curves, budgets_in, w.gains, budgets, offsets, ls) != cudaSuccess) rc = LUKV_ERR_CUDA;
+    if (cudaEventRecord(side->join, ls.st) != cudaSuccess) rc = LUKV_ERR_CUDA;
+    lc.launches += ls.launches;
+    if (rc == LUKV_OK && (launch_score_tc(dm, q_win, k, w, dev_status, all_heads(dm), true, 2, lc) != cudaSuccess ||
+                          launch_pool(dm, w.raw, w.pooled, all_heads(dm), lc) != cudaSuccess))
+      rc = LUKV_ERR_CUDA;
+    // join even after a failure: the caller's stream must not run ahead of work already enqueued
+    if (cudaStreamWaitEvent(lc.st, side->join, 0) != cudaSuccess) rc = LUKV_ERR_CUDA;
+    if (rc != LUKV_OK) return rc;
+  } else {
+    if (launch_allocate(dm, curves, budgets_in, w.gains, budgets, offsets, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+    if (run_score(dm, q_win, k, w, w.pooled, dev_status, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  }
   if (launch_select(dm, w.pooled, budgets, offsets, kept_idx, rows_cap, all_heads(dm), lc) != cudaSuccess)
     return LUKV_ERR_CUDA;
   if (launch_gather(dm, offsets, kept_idx, k, v, k_out, v_out, rows_cap, all_heads(dm), lc) != cudaSuccess)
@@ -216,7 +262,7 @@ int lukv_compress(const lukv_params_t* params, const void* q_win, const void* k,
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;
   rc = run_compress(dm, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets, rows_cap,
-                    dev_status, w, lc);
+                    dev_status, w, lc, true);
   if (rc == LUKV_OK) g_last_launches = lc.launches;
   return rc;
 }
@@ -243,7 +289,7 @@ int lukv_compress_profile(const lukv_params_t* params, const void* q_win, const 
   lc.max_events = max_times;
   cudaEventRecord(ev[0], lc.st);
   rc = run_compress(dm, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets, rows_cap,
-                    dev_status, w, lc);
+                    dev_status, w, lc, false);
   if (rc == LUKV_OK && cudaStreamSynchronize(lc.st) != cudaSuccess) rc = LUKV_ERR_CUDA;
   const int cnt = lc.launches < max_times ? lc.launches : max_times;
   if (rc == LUKV_OK) {

@@ -69,8 +69,9 @@ cudaError_t launch_lse(const Dims& dm, const float* stats, float* lse, int chunk
 // Tensor-core scorer (bf16, head_dim 128).  dev_status may be null.
 bool score_tc_supported(const Dims& dm);
 // clear_flags: zero the scorer's counters and (lse, tag) rows first (once per call, before the first range)
+// spare_sms: SMs the persistent grid leaves to kernels of other streams
 cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const Workspace& ws, int32_t* dev_status,
-                            HeadRange hr, bool clear_flags, LaunchCtx& lc);
+                            HeadRange hr, bool clear_flags, int spare_sms, LaunchCtx& lc);
 cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, HeadRange hr, LaunchCtx& lc);
 cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, float* gains,
                             int32_t* budgets, int32_t* offsets, LaunchCtx& lc);

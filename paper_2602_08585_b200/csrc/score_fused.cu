@@ -230,6 +230,10 @@ __device__ __forceinline__ float sum4(uint64_t p, uint64_t q) {
 template <int MT, int NQ>
 struct Plan {
   static_assert(MT == 1 || NQ == 2, "two query-row blocks are split over exactly two quads");
+  // An mbarrier wait only knows the parity of the phase it waits for, so the successive phases of a
+  // barrier must be waited for by the same threads in order.  Accumulator buffer b = tile % kNumBufs is
+  // read by quad tile % NQ and written by issuer tile % 2: both must be functions of b.
+  static_assert((4 / MT) % NQ == 0, "every accumulator buffer must belong to one quad");
   static constexpr int kEpiWarps = 4 * NQ;
   // + TMA producer, two MMA issuers, helper.  The count stays a multiple of 4 warps: the register
   // file is handed out as if the CTA were rounded up to one.
@@ -810,7 +814,7 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t rows) {
 }
 
 template <int MT, int NQ>
-cudaError_t launch_fused(const CUtensorMap& qm, const CUtensorMap& km, FusedArgs args, LaunchCtx& lc) {
+cudaError_t launch_fused(const CUtensorMap& qm, const CUtensorMap& km, FusedArgs args, int spare_sms, LaunchCtx& lc) {
   using P = Plan<MT, NQ>;
   const int smem = P::kTotal;
   auto kern = score_fused_kernel<MT, NQ>;
@@ -821,6 +825,7 @@ cudaError_t launch_fused(const CUtensorMap& qm, const CUtensorMap& km, FusedArgs
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
   if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, P::kThreads, smem)) != cudaSuccess) return e;
   if (per_sm < 1 || sms < 1) return cudaErrorLaunchOutOfResources;
+  if (spare_sms > 0 && sms > 8 * spare_sms) sms -= spare_sms;
   // A CTA runs pass 1 of later items before pass 2 of the current one, so a head's items must
   // not outnumber the CTAs (else a CTA would wait for partials that it is due to produce itself).
   while ((args.tiles_T + args.item_tiles - 1) / args.item_tiles > sms) ++args.item_tiles;
@@ -868,7 +873,7 @@ bool score_tc_supported(const Dims& dm) {
 }
 
 cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const Workspace& ws, int32_t* dev_status,
-                            HeadRange hr, bool clear_flags, LaunchCtx& lc) {
+                            HeadRange hr, bool clear_flags, int spare_sms, LaunchCtx& lc) {
   CUtensorMap qm, km;
   if (!make_map(&qm, q, (uint64_t)dm.heads() * dm.M) || !make_map(&km, k, (uint64_t)dm.heads() * dm.T))
     return cudaErrorInvalidValue;
@@ -900,10 +905,8 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
     const cudaError_t e = cudaMemsetAsync(ws.head_flags, 0, score_tc_flag_bytes(dm), lc.st);
     if (e != cudaSuccess) return e;
   }
-  if (dm.M > 128) return launch_fused<2, 2>(qm, km, args, lc);
-  static const int quads = env_int("LUKV_QUADS", 2, 3, 2);
-  if (quads == 3) return launch_fused<1, 3>(qm, km, args, lc);
-  return launch_fused<1, 2>(qm, km, args, lc);
+  if (dm.M > 128) return launch_fused<2, 2>(qm, km, args, spare_sms, lc);
+  return launch_fused<1, 2>(qm, km, args, spare_sms, lc);
 }
 
 }  // namespace lukv
