@@ -233,7 +233,10 @@ struct Plan {
   // An mbarrier wait only knows the parity of the phase it waits for, so the successive phases of a
   // barrier must be waited for by the same threads in order.  Accumulator buffer b = tile % kNumBufs is
   // read by quad tile % NQ and written by issuer tile % 2: both must be functions of b.
-  static_assert((4 / MT) % NQ == 0, "every accumulator buffer must belong to one quad");
+  // With three quads the buffers rotate over the quads, so "accumulator complete" has two barriers per
+  // buffer, used alternately: a quad that runs ahead then still waits on a barrier whose previous
+  // phase (eight tiles back) is long complete.
+  static_assert(NQ == 2 || (MT == 1 && NQ == 3), "two quads, or three that take the tiles in turn");
   static constexpr int kEpiWarps = 4 * NQ;
   // + TMA producer, two MMA issuers, helper.  The count stays a multiple of 4 warps: the register
   // file is handed out as if the CTA were rounded up to one.
@@ -249,10 +252,10 @@ struct Plan {
   static constexpr int kBarOff = kFinOff + kFinBufs * kFinBytes;
   static constexpr int kNumBufs = 4 / MT;              // accumulator buffers in TMEM
   static constexpr int kBufCols = 128 * MT;
-  // barriers: full[kStages], empty[kStages], qfull[kQSlots], qempty[kQSlots], tfull[kNumBufs],
+  // barriers: full[kStages], empty[kStages], qfull[kQSlots], qempty[kQSlots], tfull[2][kNumBufs],
   // tempty[kNumBufs], pub_full[NQ], pub_empty[NQ], lse_full[kMaxLag], lse_empty[kMaxLag], fin[kFinBufs]
   static constexpr int kBarFull = 0, kBarEmpty = kStages, kBarQFull = 2 * kStages, kBarQEmpty = kBarQFull + kQSlots,
-                       kBarTFull = kBarQEmpty + kQSlots, kBarTEmpty = kBarTFull + kNumBufs,
+                       kBarTFull = kBarQEmpty + kQSlots, kBarTEmpty = kBarTFull + 2 * kNumBufs,
                        kBarPubFull = kBarTEmpty + kNumBufs, kBarPubEmpty = kBarPubFull + NQ,
                        kBarLseFull = kBarPubEmpty + NQ, kBarLseEmpty = kBarLseFull + kMaxLag,
                        kBarFin = kBarLseEmpty + kMaxLag, kNumBars = kBarFin + kFinBufs;
@@ -397,6 +400,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
     }
     for (int b = 0; b < kNumBufs; ++b) {
       mbar_init(bar(P::kBarTFull, b), 1);
+      mbar_init(bar(P::kBarTFull, kNumBufs + b), 1);
       mbar_init(bar(P::kBarTEmpty, b), MT == 2 ? 8 : 4);
     }
     for (int q = 0; q < NQ; ++q) {
@@ -507,7 +511,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
             }
           }
           umma_commit(bar(P::kBarEmpty, s));     // the stage may be refilled once these MMAs have read it
-          umma_commit(bar(P::kBarTFull, buf));   // the accumulator is complete
+          umma_commit(bar(P::kBarTFull, buf + kNumBufs * (use & 1)));   // the accumulator is complete
         }
         if (!ok) break;
         umma_commit(bar(P::kBarQEmpty, slot));   // this issuer's share of the job no longer needs the query tiles
@@ -694,7 +698,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
         for (int t = 0; t < j.ntiles; ++t, ++tt) {
           if (MT == 1 && (int)(tt % NQ) != quad) continue;
           const uint32_t buf = tt % kNumBufs, use = tt / kNumBufs;
-          const bool ok = mbar_wait(bar(P::kBarTFull, buf), use & 1, abort_flag, a.dev_status);
+          const bool ok = mbar_wait(bar(P::kBarTFull, buf + kNumBufs * (use & 1)), (use >> 1) & 1, abort_flag, a.dev_status);
           if (ok) {
             tc_fence_after();
             const int j0 = (j.tile0 + t) * kTileKeys;
@@ -736,7 +740,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
         for (int t = 0; t < j.ntiles; ++t, ++tt) {
           if ((int)(tt % NQ) != quad) continue;
           const uint32_t buf = tt % kNumBufs, use = tt / kNumBufs;
-          const bool ok = mbar_wait(bar(P::kBarTFull, buf), use & 1, abort_flag, a.dev_status);
+          const bool ok = mbar_wait(bar(P::kBarTFull, buf + kNumBufs * (use & 1)), (use >> 1) & 1, abort_flag, a.dev_status);
           if (ok) {
             tc_fence_after();
             const int key = (j.tile0 + t) * kTileKeys + qtid;
@@ -906,6 +910,8 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
     if (e != cudaSuccess) return e;
   }
   if (dm.M > 128) return launch_fused<2, 2>(qm, km, args, spare_sms, lc);
+  static const int quads = env_int("LUKV_QUADS", 2, 3, 2);
+  if (quads == 3) return launch_fused<1, 3>(qm, km, args, spare_sms, lc);
   return launch_fused<1, 2>(qm, km, args, spare_sms, lc);
 }
 
