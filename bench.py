@@ -150,7 +150,7 @@ class ClockSampler(threading.Thread):
     def run(self):
         while self.ok and not self._halt.is_set():
             self.sample_once()
-            time.sleep(0.005)
+            time.sleep(0.002)
 
     def stop(self):
         self._halt.set()
@@ -196,12 +196,17 @@ def kernel_bytes(name, wl, rows):
 
 
 def load_traffic(kernel, workload):
-    """DRAM bytes per launch from a committed ncu capture, if one is recorded."""
+    """DRAM bytes per launch (read + write) from the committed ncu summary, if one is recorded there:
+    lines `traffic <workload> <kernel> <bytes>` in profiles/dram_traffic.txt."""
     try:
-        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
-            return json.load(f).get(workload, {}).get(kernel)
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            for line in f:
+                t = line.split()
+                if len(t) == 4 and t[0] == "traffic" and t[1] == workload and t[2] == kernel:
+                    return float(t[3])
     except Exception:
-        return None
+        pass
+    return None
 
 
 def run_ours(args):
@@ -280,10 +285,26 @@ def run_ours(args):
         kv["share"] = kv["ms_per_launch"] * kv["launches_per_step"] / total_kernel_ms
     dom = max(kernels, key=lambda nm: kernels[nm]["ms_per_launch"] * kernels[nm]["launches_per_step"])
     dom_bytes = kernel_bytes(dom, wl, out.rows)
-    dom_gbs = dom_bytes / (kernels[dom]["ms_per_launch"] * 1e-3) / 1e9
-    roofline = {"kernel": dom, "bound": "hbm", "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
-                "frac": dom_gbs / peak, "peak_source": peak_src, "algorithmic_bytes_per_launch": dom_bytes,
-                "traffic": load_traffic(dom, wl.name)}
+    dom_s = kernels[dom]["ms_per_launch"] * 1e-3
+    dom_gbs = dom_bytes / dom_s / 1e9
+    if dom == "score_fused":
+        # The fused scorer evaluates one exp2 per (query row, visible key) in each of its two passes on the
+        # special-function units, which do 16 per clock and SM: that, not HBM, bounds it (K crosses HBM
+        # once; the second pass reads it from L2).  Peak = 16 x SMs x max SM clock.
+        import torch
+        sms = torch.cuda.get_device_properties(local).multi_processor_count
+        exps = 2.0 * wl.S * wl.N * wl.G * wl.w * wl.T
+        peak_exp = 16.0 * sms * (sampler.max_mhz or 1965) * 1e6 / 1e9
+        roofline = {"kernel": dom, "bound": "alu", "achieved": exps / dom_s / 1e9, "peak": peak_exp,
+                    "unit": "Gexp2/s", "frac": exps / dom_s / 1e9 / peak_exp,
+                    "peak_source": "16 exp2 per clock per SM x SM count x max SM clock",
+                    "algorithmic_exp2_per_launch": exps, "algorithmic_bytes_per_launch": dom_bytes,
+                    "hbm_achieved_gbs": dom_gbs, "hbm_peak_gbs": peak, "hbm_frac": dom_gbs / peak,
+                    "hbm_peak_source": peak_src, "traffic": load_traffic(dom, wl.name)}
+    else:
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
+                    "frac": dom_gbs / peak, "peak_source": peak_src, "algorithmic_bytes_per_launch": dom_bytes,
+                    "traffic": load_traffic(dom, wl.name)}
     es = 2 if wl.dtype == "bf16" else 4
     path_bytes = wl.S * wl.N * wl.T * wl.d * es + 2 * out.rows * wl.d * es   # K read + kept K/V written
     path_gbs = path_bytes / (ms * 1e-3) / 1e9

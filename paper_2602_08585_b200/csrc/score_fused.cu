@@ -901,7 +901,7 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
   args.npad = (dm.M + 31) & ~31;
   static const int hints = env_int("LUKV_L2_HINTS", 0, 1, 1);
   args.l2_hints = hints;
-  static const int lag = env_int("LUKV_LAG", 2, kMaxLag, 3);
+  static const int lag = env_int("LUKV_LAG", 2, kMaxLag, 2);
   args.lag = lag;
   args.scale_log2 = dm.scale_log2;
   // the per-head counters and the (value, tag) rows must start at zero; they are adjacent in the workspace
