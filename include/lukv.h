@@ -15,8 +15,9 @@
  *
  * Conventions
  *   - Every pointer is DEVICE memory unless marked HOST.  The caller owns every buffer;
- *     the library allocates nothing, keeps no state between calls and never synchronises
- *     the stream.  All work is enqueued on `stream` (a cudaStream_t passed as void*).
+ *     the library allocates no device memory, keeps no results between calls and never
+ *     synchronises the stream.  All work is ordered on `stream` (a cudaStream_t passed as
+ *     void*).
  *   - Tensors are contiguous, row-major, in the layouts written next to each argument.
  *   - Notation: S sequences, L layers, H KV heads per layer, N = L*H heads per sequence,
  *     G query heads per KV head, d head dim, T context length, w observation window,
@@ -143,7 +144,12 @@ LUKV_API int lukv_select_gather(const lukv_params_t* params, const float* scores
  * intermediate scores kept in the workspace.  Arguments as above.  Returns
  * LUKV_ERR_OUTPUT_TOO_SMALL when rows_cap < sum_q B_q + S*N*w.
  *   dev_status [1] int32, may be NULL: set to 0 by the call; a kernel that gives up on a
- *   bounded wait stores LUKV_ERR_TIMEOUT there.
+ *   bounded wait stores LUKV_ERR_TIMEOUT there (the tensor-core scorer's CTAs wait for one
+ *   another; it is launched cooperatively, so this only happens if the device is taken away).
+ * The allocation kernels run on an auxiliary stream beside the scorer; that stream and two
+ * events are created on the first call on a device and kept until the process exits.  The
+ * caller's stream waits for them inside the call, so everything the call enqueues is ordered
+ * after earlier work on `stream` and before later work on it.
  */
 LUKV_API int lukv_compress(const lukv_params_t* params, const void* q_win, const void* k, const void* v,
                   const float* curves, const int64_t* budgets_in, void* k_out, void* v_out, int32_t* kept_idx,
