@@ -37,7 +37,6 @@ constexpr int kHalfBytes = kTileKeys * 128;  // one 64-channel half of a 128-row
 constexpr int kStageBytes = 2 * kHalfBytes;  // 128 keys x 128 channels bf16
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kMaxLag = 6;                   // a CTA runs pass 1 at most this many items ahead of pass 2
-constexpr int kFinBytes = 16384;             // one block of partials folded by a head's last item
 
 // ---- PTX wrappers ------------------------------------------------------------------------
 
@@ -212,6 +211,19 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// exp2 on the FMA pipe (degree-4 polynomial on the fraction, relative error 3e-6), for code that
+// must not queue behind the epilogue warps on the special-function unit.  x <= 126.
+__device__ __forceinline__ float ex2_fma(float x) {
+  x = fmaxf(x, -126.f);
+  const float t = x + 12582912.f;   // 1.5 * 2^23: the integer part of x lands in the low mantissa bits
+  const float f = x - (t - 12582912.f);  // fraction in [-0.5, 0.5]
+  float p = 0.009570101276040077f;
+  p = fmaf(p, f, 0.05591785907745361f);
+  p = fmaf(p, f, 0.240247443318367f);
+  p = fmaf(p, f, 0.6931217908859253f);
+  p = fmaf(p, f, 0.9999992847442627f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
 // both lanes of a packed pair through exp2
 __device__ __forceinline__ uint64_t ex2_pair(uint64_t x) {
   float a, b;
@@ -241,12 +253,12 @@ struct Plan {
   // + TMA producer, two MMA issuers, helper.  The count stays a multiple of 4 warps: the register
   // file is handed out as if the CTA were rounded up to one.
   static constexpr int kThreads = (kEpiWarps + 4) * 32;
-  static constexpr int kStages = MT == 1 ? 4 : 2;      // key-tile ring: a stage is held from its TMA request until the
-                                                       // MMAs that read it complete, so HBM latency needs >= 4 of them
+  static constexpr int kStages = MT == 1 ? 3 : 2;      // key-tile ring
   static constexpr int kQSlots = 2;                    // query tiles of the job in the tensor pipe and the next one
   static constexpr int kQBytes = MT * kStageBytes;     // [half][MT*128 rows][128 B]
   static constexpr int kFinBufs = 1;                   // blocks of partials in flight while a head is folded
-  static constexpr int kFinParts = kFinBytes / (128 * MT * 8);  // partials per block
+  static constexpr int kFinBytes = 16384;              // one block
+  static constexpr int kFinParts = kFinBytes / (128 * MT * 4);  // items per block (one float per row and item)
   static constexpr int kKOff = kQSlots * kQBytes;
   static constexpr int kFinOff = kKOff + kStages * kStageBytes;
   static constexpr int kBarOff = kFinOff + kFinBufs * kFinBytes;
@@ -268,13 +280,13 @@ struct Plan {
 };
 
 struct FusedArgs {
-  float* stats;        // pass 1 partials: [heads][items_per_head][128*MT] (reference, sum-exp), exp2 domain
+  float* stats;        // pass 1 partials: [heads][items_per_head][128*MT] log-sum-exp of the item's keys, exp2 domain
   float* lse;          // [heads][lse_rows] (row log-sum-exp in the exp2 domain, tag); zero at launch
   float* raw;          // pass 2 out: [heads][n]
   int* head_cnt;       // [heads] items whose partials were delivered (zero at launch)
   int32_t* dev_status;
   int M, T, w, n;
-  int lse_rows;        // M rounded up to a multiple of 2
+  int lse_rows;        // M rounded up to a multiple of 4
   int head0, nheads;   // heads [head0, head0+nheads) are scored by this launch
   int item_tiles, items_per_head, tiles_T, tiles_n;
   int npad;            // pass 2: query rows rounded up to a multiple of 32 (MMA N and columns read)
@@ -544,7 +556,8 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
           const bool ok = true;
           const Job j1 = make_job(k, false, a);
           if (ok) {
-            float2* dst = reinterpret_cast<float2*>(a.stats) + ((size_t)j1.u * a.items_per_head + j1.c) * kRowsPad;
+            // one value per row: the log-sum-exp of the item's keys, m + log2(l); -inf for an empty partial
+            float* dst = a.stats + ((size_t)j1.u * a.items_per_head + j1.c) * kRowsPad;
 #pragma unroll
             for (int rr = 0; rr < kRowsPad; rr += 32) {
               float2 v = pub_s[rr + lane];
@@ -560,7 +573,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
                   }
                 }
               }
-              dst[rr + lane] = v;  // rows beyond M carry (-inf, 0)
+              dst[rr + lane] = v.y > 0.f ? v.x + log2f(v.y) : -INFINITY;
             }
           }
           __syncwarp();
@@ -571,62 +584,85 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
           if (lane == 0 && ok && !*abort_flag) last = atom_add_acq_rel(a.head_cnt + j1.u, 1) == a.items_per_head - 1;
           last = __shfl_sync(0xffffffffu, last, 0);
           if (last) {
-            // Fold the head's partials: the bulk-copy engine brings them into shared memory in blocks of
-            // kFinParts items (one round trip per block instead of one per load); every lane folds its rows.
-            constexpr int kRowsLane = 4 * MT;
-            const char* src = reinterpret_cast<const char*>(a.stats) + (size_t)j1.u * a.items_per_head * kRowsPad * 8;
+            // Fold the head's partials into lse = log2(sum_c 2^(v_c)).  The bulk-copy engine brings them
+            // into shared memory (one round trip instead of one per load).  This warp competes with the
+            // epilogue warps for issue slots and the head's consumers wait for the result, so the fold
+            // is kept short: lane i owns rows 4i..4i+3 (one 16-byte load per item), terms are added
+            // relative to the first item's value, and the exact two-sweep form (maximum first) is only
+            // the fallback when that sum leaves a safe range.
+            constexpr int kVecs = MT;  // float4 per lane and item
+            const char* src = reinterpret_cast<const char*>(a.stats) + (size_t)j1.u * a.items_per_head * kRowsPad * 4;
             const int nblk = (a.items_per_head + P::kFinParts - 1) / P::kFinParts;
             auto request = [&](int blk) {  // lane 0
               const int parts = min(P::kFinParts, a.items_per_head - blk * P::kFinParts);
-              const uint32_t bytes = (uint32_t)parts * kRowsPad * 8, b = blk % P::kFinBufs;
-              mbar_expect_tx(bar(P::kBarFin, b), bytes);
-              bulk_load(sbase + P::kFinOff + b * kFinBytes, src + (size_t)blk * P::kFinParts * kRowsPad * 8, bytes,
-                        bar(P::kBarFin, b));
+              const uint32_t bytes = (uint32_t)parts * kRowsPad * 4;
+              mbar_expect_tx(bar(P::kBarFin, 0), bytes);
+              bulk_load(sbase + P::kFinOff, src + (size_t)blk * P::kFinParts * kRowsPad * 4, bytes, bar(P::kBarFin, 0));
             };
-            asm volatile("fence.proxy.async;" ::: "memory");
-            if (lane == 0)
-              for (int blk = 0; blk < nblk && blk < P::kFinBufs; ++blk) request(blk);
-            float fm[kRowsLane], fl[kRowsLane];
-#pragma unroll
-            for (int jj = 0; jj < kRowsLane; ++jj) fm[jj] = -INFINITY, fl[jj] = 0.f;
+            const float4* part = reinterpret_cast<const float4*>(smem + P::kFinOff);
+            float ref[kVecs][4], sum[kVecs][4];
             bool fin_ok = true;
-            for (int blk = 0; blk < nblk; ++blk) {
-              const uint32_t b = blk % P::kFinBufs;
-              fin_ok = fin_ok && mbar_wait(bar(P::kBarFin, b), fin_uses[b] & 1, abort_flag, a.dev_status);
-              ++fin_uses[b];
-              if (fin_ok) {
-                const float2* part = reinterpret_cast<const float2*>(smem + P::kFinOff + b * kFinBytes);
+            for (int pass = 0; pass < 2 && fin_ok; ++pass) {  // pass 1 only if pass 0 left the safe range
+              for (int blk = 0; blk < nblk && fin_ok; ++blk) {
+                asm volatile("fence.proxy.async;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) request(blk);
+                fin_ok = mbar_wait(bar(P::kBarFin, 0), fin_uses[0] & 1, abort_flag, a.dev_status);
+                ++fin_uses[0];
+                if (!fin_ok) break;
                 const int parts = min(P::kFinParts, a.items_per_head - blk * P::kFinParts);
-                float cm[kRowsLane], cl[kRowsLane];
+                if (blk == 0) {
 #pragma unroll
-                for (int jj = 0; jj < kRowsLane; ++jj) cm[jj] = fm[jj], cl[jj] = 0.f;
-                for (int c = 0; c < parts; ++c)
-#pragma unroll
-                  for (int jj = 0; jj < kRowsLane; ++jj) {
-                    const float2 v = part[c * kRowsPad + 32 * jj + lane];
-                    if (v.y > 0.f) cm[jj] = fmaxf(cm[jj], v.x);  // an empty partial is (-inf, 0)
+                  for (int vv = 0; vv < kVecs; ++vv) {
+                    float4 r0 = part[vv * 32 + lane];
+                    ref[vv][0] = r0.x, ref[vv][1] = r0.y, ref[vv][2] = r0.z, ref[vv][3] = r0.w;
+                    sum[vv][0] = sum[vv][1] = sum[vv][2] = sum[vv][3] = 0.f;
                   }
-                for (int c = 0; c < parts; ++c)
+                }
+                if (pass == 1 && blk == 0) {
+                  // the fallback needs the maximum of every row first; it is rare, so it simply reads the
+                  // partials from global memory
+                  const float4* g = reinterpret_cast<const float4*>(src);
+                  for (int c = 0; c < a.items_per_head; ++c)
 #pragma unroll
-                  for (int jj = 0; jj < kRowsLane; ++jj) {
-                    const float2 v = part[c * kRowsPad + 32 * jj + lane];
-                    if (v.y > 0.f) cl[jj] = fmaf(v.y, ex2(v.x - cm[jj]), cl[jj]);
-                  }
+                    for (int vv = 0; vv < kVecs; ++vv) {
+                      const float4 v = __ldcg(g + (size_t)c * (kRowsPad / 4) + vv * 32 + lane);
+                      ref[vv][0] = fmaxf(ref[vv][0], v.x), ref[vv][1] = fmaxf(ref[vv][1], v.y);
+                      ref[vv][2] = fmaxf(ref[vv][2], v.z), ref[vv][3] = fmaxf(ref[vv][3], v.w);
+                    }
+                }
+                for (int c0 = 0; c0 < parts; c0 += 8)
 #pragma unroll
-                for (int jj = 0; jj < kRowsLane; ++jj)
-                  if (cl[jj] > 0.f) {
-                    fl[jj] = fmaf(fl[jj], ex2(fm[jj] - cm[jj]), cl[jj]);
-                    fm[jj] = cm[jj];
-                  }
+                  for (int cc = 0; cc < 8; ++cc)
+                    if (c0 + cc < parts) {
+#pragma unroll
+                      for (int vv = 0; vv < kVecs; ++vv) {
+                        const float4 v = part[(c0 + cc) * (kRowsPad / 4) + vv * 32 + lane];
+                        sum[vv][0] += ex2(v.x - ref[vv][0]);
+                        sum[vv][1] += ex2(v.y - ref[vv][1]);
+                        sum[vv][2] += ex2(v.z - ref[vv][2]);
+                        sum[vv][3] += ex2(v.w - ref[vv][3]);
+                      }
+                    }
               }
-              __syncwarp();
-              if (lane == 0 && fin_ok && blk + P::kFinBufs < nblk) request(blk + P::kFinBufs);
-            }
-            float2* out = reinterpret_cast<float2*>(a.lse) + (size_t)j1.u * a.lse_rows;
+              bool safe = true;
 #pragma unroll
-            for (int jj = 0; jj < kRowsLane; ++jj) {
-              const int row = 32 * jj + lane;
-              if (row < a.lse_rows && fin_ok) __stcg(out + row, make_float2(fm[jj] + log2f(fl[jj]), 1.f));
+              for (int vv = 0; vv < kVecs; ++vv)
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (4 * (vv * 32 + lane) + e < a.M) safe = safe && (sum[vv][e] >= 1e-30f) && (sum[vv][e] <= 1e30f);
+              if (__all_sync(0xffffffffu, safe)) break;
+            }
+            float4* out = reinterpret_cast<float4*>(a.lse) + (size_t)j1.u * (a.lse_rows / 2);
+#pragma unroll
+            for (int vv = 0; vv < kVecs; ++vv) {
+              const int row = 4 * (vv * 32 + lane);
+              if (row < a.lse_rows && fin_ok) {
+                __stcg(out + row / 2, make_float4(ref[vv][0] + log2f(sum[vv][0]), 1.f, ref[vv][1] + log2f(sum[vv][1]), 1.f));
+                if (row + 2 < a.lse_rows)
+                  __stcg(out + row / 2 + 1,
+                         make_float4(ref[vv][2] + log2f(sum[vv][2]), 1.f, ref[vv][3] + log2f(sum[vv][3]), 1.f));
+              }
             }
           }
           ++kp;
@@ -869,7 +905,7 @@ size_t score_tc_stats_bytes(const Dims& dm) {
 }
 // Bytes of the block that must be zero at launch: [heads] counters, then [heads][lse_rows][2] floats.
 size_t score_tc_flag_bytes(const Dims& dm) {
-  return lse_tag_offset(dm) + (size_t)dm.heads() * ((dm.M + 1) & ~1) * 2 * sizeof(float);
+  return lse_tag_offset(dm) + (size_t)dm.heads() * ((dm.M + 3) & ~3) * 2 * sizeof(float);
 }
 
 bool score_tc_supported(const Dims& dm) {
@@ -891,7 +927,7 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
   args.T = dm.T;
   args.w = dm.w;
   args.n = dm.n;
-  args.lse_rows = (dm.M + 1) & ~1;
+  args.lse_rows = (dm.M + 3) & ~3;
   args.head0 = hr.h0;
   args.nheads = hr.nh;
   args.item_tiles = score_item_tiles();
