@@ -182,7 +182,10 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(const int32_t* _
         const int mid = (lo + hi) >> 1;
         if ((long long)__ldg(offsets + mid) <= r) lo = mid; else hi = mid;
       }
-      src_row = (long long)lo * T + __ldg(kept_idx + r);
+      // positions come from the selection kernel; clamping them keeps the copy inside the head even if
+      // the scores were not finite (their ranking is then meaningless, but nothing is read out of bounds)
+      const int pos = min(max(__ldg(kept_idx + r), 0), T - 1);
+      src_row = (long long)lo * T + pos;
     }
 #pragma unroll
     for (int b0 = 0; b0 < kBatches; b0 += kInFlight) {
