@@ -167,6 +167,16 @@ class ClockSampler(threading.Thread):
 
 # ---- our arm -------------------------------------------------------------------------------------
 
+def max_over_ranks(value, dist, device):
+    """The job-level time of a step is the slowest rank's: all-reduce MAX (no-op without a process group)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -260,10 +270,8 @@ def run_ours(args):
         sampler.sample_once()
     sampler.stop()
     ms = e0.elapsed_time(e1) / args.steps
+    ms = max_over_ranks(ms, dist, "cuda")
     if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
         dist.barrier()
     assert int(out.dev_status.item()) == 0
     tokens = wl.S * wl.T * world
@@ -335,10 +343,7 @@ def run_ours(args):
             e1.record()
             torch.cuda.synchronize()
             e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
-            if dist is not None:
-                t = torch.tensor([e2e_ms], device="cuda")
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                e2e_ms = float(t.item())
+            e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
             e2e = {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms, "steps": args.e2e_steps,
                    "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_in)),
                    "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_out))}

@@ -1,0 +1,109 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times (one fused
+lukv_compress call over the whole workload).  The oracle cannot run a whole configuration in
+reasonable time, so:
+  - allocation (budgets, offsets) is compared in full, bit for bit (the oracle's allocation is fast);
+  - a seeded sample of heads is re-drawn on the host (the generator gives identical bits on both
+    devices) and compared head by head: scores within the tolerance, kept-index agreement >= 99.9 %
+    with every mismatch at the threshold, packed bytes equal to the source rows;
+  - properties that hold at any size are checked on every head: budgets sum to B_q, offsets are the
+    running sum of budget + w, kept positions are strictly ascending inside [0, n), the window rows
+    follow, and every packed row equals the source row its index names.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_08585_b200 import lukv, synth
+from gpu_helpers import SCORE_ATOL, SCORE_RTOL, bits, params_of
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_full(oracle, name, sample_heads):
+    wl = synth.CONFIGS[name]
+    p = params_of(wl)
+    q, k, v = synth.gen_tensors(wl, "cuda")
+    curves = synth.gen_curves(wl)
+    Bs = wl.budgets()
+    ws = lukv.alloc_workspace(p)
+    out = lukv.Outputs(p, Bs)
+    lukv.lukv_compress(p, q, k, v, torch.from_numpy(curves).cuda(), Bs, out.k_out, out.v_out, out.kept_idx,
+                       out.budgets, out.offsets, out.rows, out.dev_status, ws)
+    torch.cuda.synchronize()
+    assert int(out.dev_status.item()) == 0
+    # the pooled scores of the same inputs (the fused call keeps them in its workspace)
+    scores = torch.empty((p.batch, p.N, p.n), dtype=torch.float32, device="cuda")
+    lukv.lukv_score(p, q, k, scores, ws)
+    torch.cuda.synchronize()
+
+    budgets = out.budgets.cpu().numpy()
+    offsets = out.offsets.cpu().numpy()
+    b_ref, o_ref = oracle.allocate(curves, wl.T, wl.w, Bs)
+    np.testing.assert_array_equal(budgets, b_ref)
+    np.testing.assert_array_equal(offsets, o_ref)
+    np.testing.assert_array_equal(budgets.sum(axis=1), Bs)
+    assert offsets[-1] == wl.total_rows() == out.rows
+
+    # ---- properties on every head, on the device (the tensors are large)
+    heads = wl.S * wl.N
+    bflat = out.budgets.reshape(-1).to(torch.int64)
+    off = out.offsets.to(torch.int64)
+    assert torch.equal(off[1:] - off[:-1], bflat + wl.w)
+    row_head = torch.repeat_interleave(torch.arange(heads, device="cuda"), bflat + wl.w)
+    kept = out.kept_idx.to(torch.int64)
+    rank_in_head = torch.arange(out.rows, device="cuda") - off[row_head]
+    is_win = rank_in_head >= bflat[row_head]
+    assert torch.equal(kept[is_win], (wl.n + rank_in_head - bflat[row_head])[is_win])      # window rows n..T-1
+    sel = ~is_win
+    assert int(kept[sel].min()) >= 0 and int(kept[sel].max()) < wl.n
+    same_head = row_head[1:] == row_head[:-1]
+    assert bool(torch.all((kept[1:] > kept[:-1]) | ~same_head))                              # ascending inside a head
+    src = row_head * wl.T + kept
+    kflat = k.reshape(heads * wl.T, wl.d).view(torch.int16)
+    vflat = v.reshape(heads * wl.T, wl.d).view(torch.int16)
+    step = 1 << 20
+    for r0 in range(0, out.rows, step):                                                      # packed rows are exact copies
+        r1 = min(out.rows, r0 + step)
+        assert torch.equal(out.k_out[r0:r1].view(torch.int16), kflat[src[r0:r1]])
+        assert torch.equal(out.v_out[r0:r1].view(torch.int16), vflat[src[r0:r1]])
+
+    # ---- sampled heads against the oracle
+    rng = np.random.default_rng(wl.seed)
+    sample = sorted(set(int(x) for x in rng.integers(0, heads, size=sample_heads)) | {0, heads - 1})
+    kept_np = out.kept_idx.cpu().numpy()
+    agree = total = 0
+    for u in sample:
+        qi, rem = divmod(u, wl.N)
+        layer, h = divmod(rem, wl.H)
+        qh, kh, vh = synth.gen_head(wl, qi, layer, h, "cpu")
+        assert torch.equal(kh, k[qi, layer, h].cpu())                                        # same bits on both devices
+        _, pooled = oracle.score_head(bits(qh), bits(kh), wl.kp)
+        got = scores[qi, rem].cpu().numpy()
+        err = np.abs(got.astype(np.float64) - pooled.astype(np.float64))
+        assert np.all(err <= SCORE_RTOL * np.abs(pooled.astype(np.float64)) + SCORE_ATOL), \
+            f"head {u}: worst relative error {(err / np.maximum(np.abs(pooled), 1e-300)).max():.3e}"
+        b = int(budgets.reshape(-1)[u])
+        if b == 0:
+            continue
+        ref_kept = oracle.select(pooled, b)
+        g = kept_np[offsets[u]:offsets[u] + b]
+        agree += len(np.intersect1d(g, ref_kept, assume_unique=True))
+        total += b
+        diff = np.setxor1d(g, ref_kept, assume_unique=True)
+        if len(diff):
+            t = np.sort(pooled)[::-1][b - 1].astype(np.float64)
+            gap = np.abs(pooled[diff].astype(np.float64) - t)
+            assert np.all(gap <= 2 * (SCORE_RTOL * t + SCORE_ATOL)), f"head {u}: mismatch away from the threshold"
+    assert total == 0 or agree / total >= 0.999, f"kept-index agreement {agree / max(total, 1):.5f}"
+
+
+def test_llama8b_32k_full(oracle):
+    _check_full(oracle, "llama8b_32k", sample_heads=6)
+
+
+def test_batch8_16k_mixed_full(oracle):
+    _check_full(oracle, "batch8_16k_mixed", sample_heads=6)
+
+
+def test_gqa7_128k_full(oracle):
+    _check_full(oracle, "gqa7_128k", sample_heads=2)
