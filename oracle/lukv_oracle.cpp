@@ -20,12 +20,18 @@
 //   select   : top-b positions of a head by the proxy (Sec. 4.3 "Eviction"; M^pi(k) of
 //              Sec. 3.2), ties by lower index (App. A.1 allows any fixed rule).
 //   gather   : the retained index set I of Sec. 3.2 materialised as a packed cache.
+//   profile  : offline profile = mean over calibration queries of the optimal local ratios
+//              (Sec. 4.3, Eq. "calibration_avg"); online lookup and b = floor((1-r)*n)
+//              (Sec. 4.3 "Online Execution").
 //
 // Pins (see tests, "-m not gpu"): softmax rows sum to one; closed form for identical
 // keys; single-row case against a library softmax; pooling against a library max filter;
 // PAVA against a library isotonic regression, a monotone-chain hull and the O(P^2)
 // majorant definition; greedy against exhaustive search; selection against a full sort;
-// uniform budgets against a library-op SnapKV; gather by byte equality.
+// uniform budgets against a library-op SnapKV; gather by byte equality; profile against a
+// token-by-token greedy written in the test, the closed form for identical heads, the end
+// points rho = 0 and 1, budget conservation and monotonicity in rho; lookup against a
+// hand-worked example.
 // No function here is "parity unpinned".
 //
 // Build: g++ -O2 -std=c++17 -ffp-contract=off -shared -fPIC lukv_oracle.cpp -o liblukv_oracle.so
@@ -261,6 +267,72 @@ int oracle_allocate(const float* curves, int N, int P, int T, int w, int S, cons
     for (int hid = 0; hid < N; ++hid) {
       budgets[static_cast<size_t>(q) * N + hid] = static_cast<int32_t>(b[hid]);
       running += b[hid] + w;
+      offsets[static_cast<size_t>(q) * N + hid + 1] = static_cast<int32_t>(running);
+    }
+  }
+  return 0;
+}
+
+// Offline profile aggregation (Sec. 4.3 "Profile Aggregation", Eq. "calibration_avg").
+// curves: [Mq][N][P], one set of per-head utility curves per calibration query, taken on a
+// calibration context of T tokens (n = T-w rankable).  ratios: [R] global compression
+// ratios rho in [0,1].  For every query and every rho the relaxed problem is solved for the
+// global budget B(rho) = floor((1-rho)*N*n); the query's optimal local ratio of head hid is
+// r* = 1 - b_hid/n; the profile is the mean of r* over the queries.
+// profile: [R][N], fp64 mean rounded once to fp32.  Returns 0, or -1 for a ratio outside [0,1].
+int oracle_profile_build(const float* curves, int Mq, int N, int P, int T, int w, const float* ratios, int R,
+                         float* profile) {
+  const int64_t n = T - w;
+  std::vector<int64_t> B(R);
+  for (int j = 0; j < R; ++j) {
+    const double rho = static_cast<double>(ratios[j]);
+    if (!(rho >= 0.0 && rho <= 1.0)) return -1;
+    B[j] = static_cast<int64_t>(std::floor((1.0 - rho) * static_cast<double>(static_cast<int64_t>(N) * n)));
+  }
+  std::vector<double> acc(static_cast<size_t>(R) * N, 0.0);
+  std::vector<int32_t> b(static_cast<size_t>(R) * N), off(static_cast<size_t>(R) * N + 1);
+  for (int i = 0; i < Mq; ++i) {
+    const float* ci = curves + static_cast<size_t>(i) * N * P;
+    if (oracle_allocate(ci, N, P, T, w, R, B.data(), b.data(), off.data()) != 0) return -1;
+    for (size_t e = 0; e < acc.size(); ++e) acc[e] += 1.0 - static_cast<double>(b[e]) / static_cast<double>(n);
+  }
+  for (size_t e = 0; e < acc.size(); ++e) profile[e] = static_cast<float>(acc[e] / static_cast<double>(Mq));
+  return 0;
+}
+
+// Online lookup and budgeting (Sec. 4.3 "Online Execution", steps 1-2).  profile: [R][N] over
+// the strictly ascending grid ratios[R]; sigma: [S] target global ratio of each sequence,
+// inside [ratios[0], ratios[R-1]].  Lookup: the profile row at sigma; between two grid points
+// the two neighbouring rows are interpolated linearly (at a grid point this is the row
+// itself).  Budgeting: b = floor((1-r)*n) on the n = T-w rankable positions of the new
+// context, all in fp64.  offsets: exclusive scan of (b + w) in head order.
+// Returns 0, or -1 when a sigma lies outside the grid or the grid is not ascending.
+int oracle_profile_budgets(const float* profile, const float* ratios, int R, int N, int T, int w,
+                           const float* sigma, int S, int32_t* budgets, int32_t* offsets) {
+  const int64_t n = T - w;
+  for (int j = 0; j + 1 < R; ++j)
+    if (!(ratios[j] < ratios[j + 1])) return -1;
+  int64_t running = 0;
+  offsets[0] = 0;
+  for (int q = 0; q < S; ++q) {
+    const float sg = sigma[q];
+    if (!(sg >= ratios[0] && sg <= ratios[R - 1])) return -1;
+    int j = 0;
+    while (j + 1 < R && ratios[j + 1] <= sg) ++j;  // largest j with ratios[j] <= sigma
+    const int j1 = j + 1 < R ? j + 1 : j;
+    const double t = j1 == j ? 0.0
+                             : (static_cast<double>(sg) - static_cast<double>(ratios[j])) /
+                                   (static_cast<double>(ratios[j1]) - static_cast<double>(ratios[j]));
+    for (int hid = 0; hid < N; ++hid) {
+      const double r0 = static_cast<double>(profile[static_cast<size_t>(j) * N + hid]);
+      const double r1 = static_cast<double>(profile[static_cast<size_t>(j1) * N + hid]);
+      const double r = r0 + (r1 - r0) * t;
+      double bf = std::floor((1.0 - r) * static_cast<double>(n));
+      if (bf < 0.0) bf = 0.0;
+      if (bf > static_cast<double>(n)) bf = static_cast<double>(n);
+      const int64_t bq = static_cast<int64_t>(bf);
+      budgets[static_cast<size_t>(q) * N + hid] = static_cast<int32_t>(bq);
+      running += bq + w;
       offsets[static_cast<size_t>(q) * N + hid + 1] = static_cast<int32_t>(running);
     }
   }

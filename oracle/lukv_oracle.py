@@ -38,6 +38,8 @@ def lib() -> ctypes.CDLL:
         _lib = ctypes.CDLL(_LIB)
         _lib.oracle_allocate.restype = ctypes.c_int
         _lib.oracle_compress.restype = ctypes.c_int
+        _lib.oracle_profile_build.restype = ctypes.c_int
+        _lib.oracle_profile_budgets.restype = ctypes.c_int
     return _lib
 
 
@@ -167,3 +169,31 @@ def compress(q, k, v, curves, budgets_in, G: int, kp: int, scale: float = 0.0):
     if rc != 0:
         raise ValueError("budget outside [0, N*(T-w)]")
     return out
+
+
+def profile_build(curves, T: int, w: int, ratios):
+    """Offline profile (Sec. 4.3, Eq. "calibration_avg"). curves [Mq][N][P] -> profile [R][N] fp32."""
+    curves = _c(curves, np.float32)
+    ratios = _c(ratios, np.float32)
+    Mq, N, P = curves.shape
+    R = ratios.shape[0]
+    profile = np.empty((R, N), np.float32)
+    rc = lib().oracle_profile_build(_p(curves), Mq, N, P, T, w, _p(ratios), R, _p(profile))
+    if rc != 0:
+        raise ValueError("ratio outside [0, 1]")
+    return profile
+
+
+def profile_budgets(profile, ratios, T: int, w: int, sigma):
+    """Online lookup + budgeting (Sec. 4.3). Returns (budgets [S][N] int32, offsets [S*N+1] int32)."""
+    profile = _c(profile, np.float32)
+    ratios = _c(ratios, np.float32)
+    sigma = _c(sigma, np.float32).reshape(-1)
+    R, N = profile.shape
+    S = sigma.shape[0]
+    budgets = np.empty((S, N), np.int32)
+    offsets = np.empty(S * N + 1, np.int32)
+    rc = lib().oracle_profile_budgets(_p(profile), _p(ratios), R, N, T, w, _p(sigma), S, _p(budgets), _p(offsets))
+    if rc != 0:
+        raise ValueError("sigma outside the ratio grid, or grid not strictly ascending")
+    return budgets, offsets
