@@ -48,7 +48,7 @@ typedef enum lukv_status {
   LUKV_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, flags != 0           */
   LUKV_ERR_UNSUPPORTED = -2,         /* d not in {64,128}, unknown dtype, even kp, (P-1) does  */
                                      /* not divide T, G*w > 256, P > 4097, sizes beyond int32  */
-  LUKV_ERR_BUDGET = -3,              /* some B_q < 0 or B_q > N*n                              */
+  LUKV_ERR_BUDGET = -3,              /* some B_q < 0 or B_q > N*n; a ratio outside its range   */
   LUKV_ERR_WORKSPACE_TOO_SMALL = -4, /* ws_bytes < lukv_workspace_bytes()                      */
   LUKV_ERR_OUTPUT_TOO_SMALL = -5,    /* rows_cap < sum_q B_q + S*N*w                           */
   LUKV_ERR_CUDA = -6,                /* a launch failed; cudaGetLastError() is left set        */
@@ -195,6 +195,54 @@ LUKV_API int lukv_compress_profile(const lukv_params_t* params, const void* q_wi
  */
 LUKV_API int lukv_allocate_static(const lukv_params_t* params, const float* curves, const int64_t* budgets_in,
                                   int32_t* budgets, int32_t* offsets, void* stream);
+
+/*
+ * Offline profile (Sec. 4.3 "Offline Optimal Budget Estimation", Eq. "calibration_avg").
+ * Input: the per-head utility curves of n_queries calibration queries on one calibration
+ * context (the paper uses about 4,000 tokens and 30 queries) and a grid of n_ratios global
+ * compression ratios.  For every query and every grid ratio rho the relaxed allocation
+ * problem of stage (b) is solved for the global budget B(rho) = floor((1-rho)*N*n), n = T-w
+ * being the rankable positions of the calibration context; the query's optimal local ratio
+ * of head hid is r* = 1 - b_hid/n; the profile entry is the mean of r* over the queries
+ * (fp64, rounded once to fp32).  Token resolution is P = T+1 (s = 1).
+ *
+ *   calib     the calibration shape: n_layers, n_kv_heads, ctx_len, window, curve_points as
+ *             in stage (b); batch must be 1; the other fields must be valid but are unused
+ *   curves    [n_queries][N][P] fp32
+ *   ratios    [n_ratios] fp32, HOST   each in [0,1] (else LUKV_ERR_BUDGET); read before
+ *             the call returns
+ *   profile   [n_ratios][N] fp32      out; 0 = keep everything, 1 = evict everything
+ *   ws        lukv_profile_workspace_bytes() bytes, 256-byte aligned
+ * Limits: N*n_ratios*T < 2^31, n_queries*N*P < 2^31, n_queries <= 65535.
+ */
+LUKV_API int lukv_profile_workspace_bytes(const lukv_params_t* calib, int32_t n_queries, int32_t n_ratios,
+                                          size_t* bytes /* HOST, out */);
+LUKV_API int lukv_profile_build(const lukv_params_t* calib, const float* curves, int32_t n_queries,
+                                const float* ratios, int32_t n_ratios, float* profile, void* ws, size_t ws_bytes,
+                                void* stream);
+
+/*
+ * Online lookup and budgeting (Sec. 4.3 "Online Execution", steps 1 and 2), the paper's
+ * deployment front end in place of lukv_allocate: sequence q with target global compression
+ * ratio sigma[q] takes the profile row at sigma[q] -- linearly interpolated between the two
+ * neighbouring grid rows when sigma[q] is not a grid point (the paper leaves that case
+ * open) -- and every head gets b = floor((1-r)*n), n = T-w of the NEW context described by
+ * `params`, clamped to [0,n]; all in fp64.  The budgets of a sequence add up to at most
+ * (1-sigma)*N*n and miss it by less than one token per head (plus the fp32 rounding of the
+ * profile); unlike lukv_allocate the sum is not exact.  Step 3 (eviction) is
+ * lukv_score followed by lukv_select_gather with these budgets and offsets.
+ *
+ *   profile   [n_ratios][N] fp32       as produced by lukv_profile_build (same N)
+ *   ratios    [n_ratios] fp32, HOST    strictly ascending (else LUKV_ERR_INVALID_ARG)
+ *   sigma     [S] fp32, HOST           ratios[0] <= sigma[q] <= ratios[n_ratios-1]
+ *                                      (else LUKV_ERR_BUDGET); both read before return
+ *   budgets   [S][N] int32             out
+ *   offsets   [S*N+1] int32            out: exclusive scan of (budgets + w); the total row
+ *                                      count offsets[S*N] is at most S*N*T
+ */
+LUKV_API int lukv_profile_budgets(const lukv_params_t* params, const float* profile, const float* ratios,
+                                  int32_t n_ratios, const float* sigma, int32_t* budgets, int32_t* offsets,
+                                  void* stream);
 
 /* Static description of a status code. */
 LUKV_API const char* lukv_strerror(int code);

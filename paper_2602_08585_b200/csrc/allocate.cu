@@ -91,6 +91,10 @@ struct GreedyArgs {
   int seq0;                           // first sequence of this launch
 };
 
+struct SetStride {
+  size_t gains, budgets, offsets;  // elements between consecutive curve sets
+};
+
 // Sort key of segment (hid,k): ascending key order == greedy consumption order.
 __device__ __forceinline__ unsigned long long seg_key(float gain, unsigned k, unsigned hid, unsigned N) {
   return ((unsigned long long)(~__float_as_uint(gain)) << 32) | (unsigned long long)(k * N + hid);
@@ -107,10 +111,17 @@ __device__ __forceinline__ long long capsum(int c, int seg, int n) {  // tokens 
 // active segments weighted by capacity, picks the byte at which the remaining budget runs
 // out and narrows every head's range to it.  Keys are unique, so one segment remains: the
 // partially bought one.  `tph` threads (a power of two) share a head and split its range.
+//
+// blockIdx.y selects one of several independent curve sets (the calibration queries of the
+// offline profile, which share the budgets): set i reads gains + i*set.gains, writes
+// budgets + i*set.budgets and offsets + i*set.offsets.  The hot path launches one set.
 __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __restrict__ gains, GreedyArgs args,
                                                                 int32_t* __restrict__ budgets,
-                                                                int32_t* __restrict__ offsets, int N, int P, int seg,
-                                                                int nseg, int n, int w, int tph) {
+                                                                int32_t* __restrict__ offsets, SetStride set, int N,
+                                                                int P, int seg, int nseg, int n, int w, int tph) {
+  gains += (size_t)blockIdx.y * set.gains;
+  budgets += (size_t)blockIdx.y * set.budgets;
+  offsets += (size_t)blockIdx.y * set.offsets;
   extern __shared__ __align__(16) unsigned char greedy_smem[];
   int* lo = reinterpret_cast<int*>(greedy_smem);  // [N]
   int* hi = lo + N;                               // [N]
@@ -280,24 +291,31 @@ __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __r
 
 }  // namespace
 
-cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, float* gains,
-                            int32_t* budgets, int32_t* offsets, LaunchCtx& lc) {
-  cudaStream_t st = lc.st;
-  // hull: one warp per head, up to 4 warps per block (12 bytes of shared memory per curve point and warp)
-  int hw = (int)((200u * 1024u) / hull_bytes_per_warp(dm.P));
+cudaError_t launch_hull(const float* curves, float* gains, int64_t n_curves, int P, LaunchCtx& lc) {
+  // one warp per curve, up to 4 warps per block (12 bytes of shared memory per curve point and warp)
+  int hw = (int)((200u * 1024u) / hull_bytes_per_warp(P));
   hw = hw > 4 ? 4 : (hw < 1 ? 1 : hw);
-  const size_t hull_smem = hull_bytes_per_warp(dm.P) * hw;
+  const size_t hull_smem = hull_bytes_per_warp(P) * hw;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(hull_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hull_smem)) != cudaSuccess)
     return e;
-  hull_kernel<<<(dm.N + hw - 1) / hw, hw * 32, hull_smem, st>>>(curves, gains, dm.N, dm.P);
+  hull_kernel<<<(unsigned)((n_curves + hw - 1) / hw), hw * 32, hull_smem, lc.st>>>(curves, gains, (int)n_curves, P);
   lc.mark("hull");
+  return cudaGetLastError();
+}
 
+cudaError_t launch_greedy(const Dims& dm, const float* gains, const int64_t* budgets_host, int32_t* budgets,
+                          int32_t* offsets, int n_sets, LaunchCtx& lc) {
+  cudaError_t e;
   const size_t greedy_smem = (size_t)dm.N * 4 * sizeof(int);
   int tph = 1;  // threads per head: the largest power of two <= 1024/N, at most 32
   while (tph < 32 && tph * 2 * dm.N <= kGreedyThreads) tph *= 2;
   if ((e = cudaFuncSetAttribute(greedy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)greedy_smem)) != cudaSuccess)
     return e;
+  SetStride set;
+  set.gains = (size_t)dm.N * (dm.P - 1);
+  set.budgets = (size_t)dm.S * dm.N;
+  set.offsets = (size_t)dm.S * dm.N + 1;
   long long base = 0;
   for (int q0 = 0; q0 < dm.S; q0 += kSeqPerLaunch) {
     GreedyArgs args;
@@ -312,11 +330,18 @@ cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* 
       base += budgets_host[q0 + i] + (long long)dm.N * dm.w;
     }
     args.seq0 = q0;
-    greedy_kernel<<<cnt, kGreedyThreads, greedy_smem, st>>>(gains, args, budgets, offsets, dm.N, dm.P, dm.seg, dm.nseg,
-                                                            dm.n, dm.w, tph);
+    greedy_kernel<<<dim3(cnt, n_sets), kGreedyThreads, greedy_smem, lc.st>>>(gains, args, budgets, offsets, set, dm.N,
+                                                                             dm.P, dm.seg, dm.nseg, dm.n, dm.w, tph);
     lc.mark("greedy");
   }
   return cudaGetLastError();
+}
+
+cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, float* gains,
+                            int32_t* budgets, int32_t* offsets, LaunchCtx& lc) {
+  cudaError_t e = launch_hull(curves, gains, dm.N, dm.P, lc);
+  if (e != cudaSuccess) return e;
+  return launch_greedy(dm, gains, budgets_host, budgets, offsets, 1, lc);
 }
 
 }  // namespace lukv

@@ -349,12 +349,125 @@ int lukv_allocate_static(const lukv_params_t* params, const float* curves, const
   return LUKV_OK;
 }
 
+// ---- offline profile and online lookup (Sec. 4.3) -----------------------------------------
+
+namespace {
+struct ProfileWs {
+  float* gains;      // [Mq][N][P-1]
+  int32_t* budgets;  // [Mq][R][N]
+  int32_t* offsets;  // [Mq][R*N+1] (written by the greedy kernel, not used further)
+  size_t bytes;
+};
+ProfileWs carve_profile_ws(const Dims& dm, int n_queries, void* base) {
+  ProfileWs ws;
+  char* p = static_cast<char*>(base);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    void* r = p ? p + off : nullptr;
+    off += align256(bytes);
+    return r;
+  };
+  const size_t Mq = (size_t)n_queries, RN = (size_t)dm.S * dm.N;
+  ws.gains = static_cast<float*>(take(Mq * dm.N * (dm.P - 1) * sizeof(float)));
+  ws.budgets = static_cast<int32_t*>(take(Mq * RN * sizeof(int32_t)));
+  ws.offsets = static_cast<int32_t*>(take(Mq * (RN + 1) * sizeof(int32_t)));
+  ws.bytes = off;
+  return ws;
+}
+// Dims of the calibration problem: the n_ratios grid points take the place of the sequences.
+int make_profile_dims(const lukv_params_t* calib, int32_t n_queries, int32_t n_ratios, Dims* dm) {
+  if (!calib || n_queries < 1 || n_ratios < 1 || calib->batch != 1) return LUKV_ERR_INVALID_ARG;
+  lukv_params_t p = *calib;
+  p.batch = n_ratios;
+  const int rc = make_dims(&p, dm);
+  if (rc != LUKV_OK) return rc;
+  if ((int64_t)n_queries * dm->N * (int64_t)dm->P >= (int64_t)1 << 31 || n_queries > 65535) return LUKV_ERR_UNSUPPORTED;
+  return LUKV_OK;
+}
+}  // namespace
+
+int lukv_profile_workspace_bytes(const lukv_params_t* calib, int32_t n_queries, int32_t n_ratios, size_t* bytes) {
+  Dims dm;
+  if (!bytes) return LUKV_ERR_INVALID_ARG;
+  const int rc = make_profile_dims(calib, n_queries, n_ratios, &dm);
+  if (rc != LUKV_OK) return rc;
+  *bytes = carve_profile_ws(dm, n_queries, nullptr).bytes;
+  return LUKV_OK;
+}
+
+int lukv_profile_build(const lukv_params_t* calib, const float* curves, int32_t n_queries, const float* ratios,
+                       int32_t n_ratios, float* profile, void* ws, size_t ws_bytes, void* stream) {
+  Dims dm;
+  int rc = make_profile_dims(calib, n_queries, n_ratios, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (!curves || !ratios || !profile || !ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return LUKV_ERR_INVALID_ARG;
+  const ProfileWs w = carve_profile_ws(dm, n_queries, ws);
+  if (ws_bytes < w.bytes) return LUKV_ERR_WORKSPACE_TOO_SMALL;
+  // global budget of every grid point: B(rho) = floor((1 - rho) * N * n)
+  int64_t* B = static_cast<int64_t*>(malloc(sizeof(int64_t) * (size_t)n_ratios));
+  if (!B) return LUKV_ERR_CUDA;
+  for (int j = 0; j < n_ratios; ++j) {
+    const double rho = (double)ratios[j];
+    if (!(rho >= 0.0 && rho <= 1.0)) {
+      free(B);
+      return LUKV_ERR_BUDGET;
+    }
+    B[j] = (int64_t)floor((1.0 - rho) * (double)((int64_t)dm.N * dm.n));
+  }
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  cudaError_t e = launch_hull(curves, w.gains, (int64_t)n_queries * dm.N, dm.P, lc);
+  if (e == cudaSuccess) e = launch_greedy(dm, w.gains, B, w.budgets, w.offsets, n_queries, lc);
+  free(B);  // the budgets travel by value in the launch arguments
+  if (e == cudaSuccess) e = launch_profile_mean(w.budgets, profile, n_queries, (int64_t)dm.S * dm.N, dm.n, lc);
+  if (e != cudaSuccess) return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
+}
+
+int lukv_profile_budgets(const lukv_params_t* params, const float* profile, const float* ratios, int32_t n_ratios,
+                         const float* sigma, int32_t* budgets, int32_t* offsets, void* stream) {
+  Dims dm;
+  int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (!profile || !ratios || !sigma || !budgets || !offsets || n_ratios < 1) return LUKV_ERR_INVALID_ARG;
+  for (int j = 0; j + 1 < n_ratios; ++j)
+    if (!(ratios[j] < ratios[j + 1])) return LUKV_ERR_INVALID_ARG;
+  const size_t S = (size_t)dm.S;
+  int* rows = static_cast<int*>(malloc(S * (2 * sizeof(int) + sizeof(double))));
+  if (!rows) return LUKV_ERR_CUDA;
+  int* row_lo = rows;
+  int* row_hi = rows + S;
+  double* frac = reinterpret_cast<double*>(rows + 2 * S);
+  for (int q = 0; q < dm.S; ++q) {
+    const float sg = sigma[q];
+    if (!(sg >= ratios[0] && sg <= ratios[n_ratios - 1])) {
+      free(rows);
+      return LUKV_ERR_BUDGET;
+    }
+    int j = 0;
+    while (j + 1 < n_ratios && ratios[j + 1] <= sg) ++j;
+    const int j1 = j + 1 < n_ratios ? j + 1 : j;
+    row_lo[q] = j;
+    row_hi[q] = j1;
+    frac[q] = j1 == j ? 0.0 : ((double)sg - (double)ratios[j]) / ((double)ratios[j1] - (double)ratios[j]);
+  }
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  const cudaError_t e =
+      launch_profile_budgets(profile, row_lo, row_hi, frac, dm.S, dm.N, dm.n, dm.w, budgets, offsets, lc);
+  free(rows);
+  if (e != cudaSuccess) return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
+}
+
 const char* lukv_strerror(int code) {
   switch (code) {
     case LUKV_OK: return "ok";
     case LUKV_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, non-positive size, flags != 0)";
     case LUKV_ERR_UNSUPPORTED: return "unsupported configuration (head_dim, dtype, even pool kernel, curve grid, G*w > 256 or sizes beyond 32 bits)";
-    case LUKV_ERR_BUDGET: return "budget outside [0, N*(T-w)]";
+    case LUKV_ERR_BUDGET: return "budget outside [0, N*(T-w)], or a compression ratio outside its range";
     case LUKV_ERR_WORKSPACE_TOO_SMALL: return "workspace smaller than lukv_workspace_bytes()";
     case LUKV_ERR_OUTPUT_TOO_SMALL: return "rows_cap smaller than sum(B_q) + S*N*w";
     case LUKV_ERR_CUDA: return "CUDA launch failed";

@@ -75,6 +75,18 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
 cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, HeadRange hr, LaunchCtx& lc);
 cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, float* gains,
                             int32_t* budgets, int32_t* offsets, LaunchCtx& lc);
+// The two halves of launch_allocate.  launch_hull treats its input as n_curves independent curves;
+// launch_greedy solves n_sets curve sets (gains [n_sets][N][P-1]) for the same dm.S budgets and
+// writes budgets [n_sets][S][N] and offsets [n_sets][S*N+1].
+cudaError_t launch_hull(const float* curves, float* gains, int64_t n_curves, int P, LaunchCtx& lc);
+cudaError_t launch_greedy(const Dims& dm, const float* gains, const int64_t* budgets_host, int32_t* budgets,
+                          int32_t* offsets, int n_sets, LaunchCtx& lc);
+// Offline profile (mean of the local ratios) and online lookup + budgeting.
+cudaError_t launch_profile_mean(const int32_t* budgets, float* profile, int n_queries, int64_t count, int n,
+                                LaunchCtx& lc);
+constexpr int kLookupSeqPerLaunch = 32;
+cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, const int* row_hi, const double* frac,
+                                   int S, int N, int n, int w, int32_t* budgets, int32_t* offsets, LaunchCtx& lc);
 cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* budgets, const int32_t* offsets,
                           int32_t* kept_idx, int64_t rows_cap, HeadRange hr, LaunchCtx& lc);
 cudaError_t launch_gather(const Dims& dm, const int32_t* offsets, const int32_t* kept_idx, const void* k,

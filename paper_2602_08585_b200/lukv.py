@@ -21,7 +21,8 @@ ERR_OUTPUT_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 
 EXPORTS = ("lukv_workspace_bytes", "lukv_score", "lukv_allocate", "lukv_select_gather", "lukv_compress",
-           "lukv_strerror", "lukv_last_launch_count", "lukv_compress_profile", "lukv_allocate_static")
+           "lukv_strerror", "lukv_last_launch_count", "lukv_compress_profile", "lukv_allocate_static",
+           "lukv_profile_workspace_bytes", "lukv_profile_build", "lukv_profile_budgets")
 
 
 class Params(ctypes.Structure):
@@ -72,6 +73,9 @@ def lib() -> ctypes.CDLL:
         L.lukv_compress_profile.argtypes = L.lukv_compress.argtypes + [ctypes.POINTER(KernelTime), ctypes.c_int,
                                                                        ctypes.POINTER(ctypes.c_int)]
         L.lukv_allocate_static.argtypes = [pp, vp, vp, vp, vp, vp]
+        L.lukv_profile_workspace_bytes.argtypes = [pp, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(sz)]
+        L.lukv_profile_build.argtypes = [pp, vp, ctypes.c_int32, vp, ctypes.c_int32, vp, vp, sz, vp]
+        L.lukv_profile_budgets.argtypes = [pp, vp, vp, ctypes.c_int32, vp, vp, vp, vp]
         L.lukv_strerror.argtypes = [ctypes.c_int]
         L.lukv_strerror.restype = ctypes.c_char_p
         for name in EXPORTS[:5] + EXPORTS[6:]:
@@ -148,6 +152,39 @@ def lukv_allocate_static(params: Params, curves, budgets_in, budgets, offsets, s
     rc = lib().lukv_allocate_static(ctypes.byref(params), _ptr(curves), b.ctypes.data, _ptr(budgets), _ptr(offsets),
                                     _stream(stream))
     return _check(rc, "lukv_allocate_static", check)
+
+
+def _host_f32(x) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(x, dtype=np.float32).reshape(-1))
+
+
+def lukv_profile_workspace_bytes(calib: Params, n_queries: int, n_ratios: int) -> int:
+    out = ctypes.c_size_t(0)
+    rc = lib().lukv_profile_workspace_bytes(ctypes.byref(calib), int(n_queries), int(n_ratios), ctypes.byref(out))
+    if rc != OK:
+        raise LukvError(rc, "lukv_profile_workspace_bytes")
+    return int(out.value)
+
+
+def lukv_profile_build(calib: Params, curves, n_queries: int, ratios, profile, ws, stream=None,
+                       check: bool = True) -> int:
+    """Offline profile: curves [n_queries][N][P] (device), ratios (host) -> profile [len(ratios)][N] (device)."""
+    r = _host_f32(ratios)
+    rc = lib().lukv_profile_build(ctypes.byref(calib), _ptr(curves), int(n_queries), r.ctypes.data, int(r.shape[0]),
+                                  _ptr(profile), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                  _stream(stream))
+    return _check(rc, "lukv_profile_build", check)
+
+
+def lukv_profile_budgets(params: Params, profile, ratios, sigma, budgets, offsets, stream=None,
+                         check: bool = True) -> int:
+    """Online lookup + budgeting: profile (device), ratios and per-sequence sigma (host) -> budgets, offsets."""
+    r, sg = _host_f32(ratios), _host_f32(sigma)
+    if sg.shape[0] != params.batch:
+        raise ValueError("one target ratio per sequence")
+    rc = lib().lukv_profile_budgets(ctypes.byref(params), _ptr(profile), r.ctypes.data, int(r.shape[0]),
+                                    sg.ctypes.data, _ptr(budgets), _ptr(offsets), _stream(stream))
+    return _check(rc, "lukv_profile_budgets", check)
 
 
 def lukv_select_gather(params: Params, scores, budgets, offsets, k, v, k_out, v_out, kept_idx, rows_cap: int, ws,

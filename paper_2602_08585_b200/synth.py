@@ -30,6 +30,7 @@ BASE_SEED = 20260208
 
 # tensor ids
 _TID_Q, _TID_K, _TID_V, _TID_NEEDLE_POS, _TID_NEEDLE_NOISE, _TID_OUTLIER, _TID_CURVE_E, _TID_CURVE_B = range(1, 9)
+_TID_CALIB_HEAD, _TID_CALIB_E = 9, 10
 
 
 @dataclass(frozen=True)
@@ -269,6 +270,30 @@ def gen_curves(wl: Workload, concave: bool = False) -> np.ndarray:
         if concave:
             inc = np.sort(inc)[::-1]
         out[hid, 1:] = np.cumsum(inc).astype(np.float32)
+    return out
+
+
+def gen_calibration_curves(seed: int, n_queries: int, N: int, T: int) -> np.ndarray:
+    """Token-resolution utility curves [n_queries][N][T+1] float32 of a calibration context of T tokens,
+    one set per calibration query (the inputs of the offline profile; the paper's default
+    calibration set is a context of about 4,000 tokens with 30 queries).
+
+    Each head has a decay exponent in [0.2, 1.6] and a scale in [0.25, 4] that all queries
+    share, which gives the heads the consistent preference across queries that the profile
+    averages over; the increment of token k is scale * (k+1)^-exponent times an Exp(1) draw
+    per (query, head, token), so single curves are noisy and non-concave.
+    """
+    out = np.zeros((n_queries, N, T + 1), dtype=np.float32)
+    k = np.arange(1, T + 1, dtype=np.float64)
+    for hid in range(N):
+        hh = _hash_u32_host(seed, _TID_CALIB_HEAD, hid, 2).astype(np.float64) / 4294967296.0
+        alpha = 0.2 + 1.4 * hh[0]
+        scale = 0.25 * 16.0 ** hh[1]
+        trend = scale * k ** (-alpha)
+        for i in range(n_queries):
+            he = _hash_u32_host(seed, _TID_CALIB_E, i * N + hid, T).astype(np.float64)
+            inc = -np.log1p(-(he + 0.5) / 4294967296.0) * trend
+            out[i, hid, 1:] = np.cumsum(inc).astype(np.float32)
     return out
 
 

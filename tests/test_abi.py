@@ -103,3 +103,21 @@ def test_binding_fails_loudly_without_the_library(monkeypatch):
     monkeypatch.setattr(lukv, "LIB_PATH", "/nonexistent/liblukv.so")
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         lukv.lib()
+
+
+def test_profile_argument_errors_come_back_before_any_launch():
+    calib = _p(T=256, P=257)
+    f = _Fake()
+    grid = [0.0, 0.5, 1.0]
+    assert lukv.lukv_profile_workspace_bytes(calib, 3, 5) > 0
+    assert lukv.lukv_profile_workspace_bytes(calib, 6, 5) > lukv.lukv_profile_workspace_bytes(calib, 3, 5)
+    assert lukv.lukv_profile_build(calib, f, 2, grid, f, _Fake(nbytes=16), check=False) == lukv.ERR_WORKSPACE_TOO_SMALL
+    assert lukv.lukv_profile_build(calib, f, 2, [0.5, 1.5], f, f, check=False) == lukv.ERR_BUDGET
+    assert lukv.lukv_profile_build(calib, f, 0, grid, f, f, check=False) == lukv.ERR_INVALID_ARG
+    assert lukv.lukv_profile_build(calib, None, 2, grid, f, f, check=False) == lukv.ERR_INVALID_ARG
+    assert lukv.lukv_profile_build(_p(S=2, T=256, P=257), f, 2, grid, f, f, check=False) == lukv.ERR_INVALID_ARG
+    p = _p(S=2)
+    assert lukv.lukv_profile_budgets(p, f, [0.5, 0.5], [0.5, 0.5], f, f, check=False) == lukv.ERR_INVALID_ARG
+    assert lukv.lukv_profile_budgets(p, f, grid, [0.5, 1.25], f, f, check=False) == lukv.ERR_BUDGET
+    assert lukv.lukv_profile_budgets(p, f, [0.2, 0.8], [0.1, 0.5], f, f, check=False) == lukv.ERR_BUDGET
+    assert lukv.lukv_profile_budgets(p, None, grid, [0.5, 0.5], f, f, check=False) == lukv.ERR_INVALID_ARG
