@@ -38,6 +38,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_32k")
+    ap.add_argument("--path", default="compress", choices=["compress", "profile"],
+                    help="compress: the headline path; profile: the offline profile build and the online "
+                         "lookup front end (secondary measurement, single GPU)")
     ap.add_argument("--layers", type=int, default=0,
                     help="override the workload's layer count (a reduced case for profiler captures)")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -381,6 +384,98 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_profile_path(args):
+    """Secondary measurement (Sec. 4.3): the offline profile build at the paper's default calibration size
+    (30 queries, a 4,000-token context, token-resolution curves, ratios 0.01..0.99) and the online mode
+    (lookup + budgeting, scoring, selection, gather) on the headline workload."""
+    import time
+    import numpy as np
+    import torch
+    from paper_2602_08585_b200 import lukv, synth
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (the path has no CPU fallback)"
+    torch.cuda.set_device(0)
+    lukv.lib()
+    wl = pick_workload(args)
+    Mq, Tc, R = 30, 4000, 99
+    ratios = (np.arange(1, R + 1) / 100.0).astype(np.float32)
+    calib = lukv.make_params(1, wl.L, wl.H, 1, 64, Tc, wl.w, 1, "fp32", Tc + 1)
+    U_np = synth.gen_calibration_curves(synth.BASE_SEED, Mq, wl.N, Tc)
+    U = torch.from_numpy(U_np).cuda()
+    pws = torch.empty(lukv.lukv_profile_workspace_bytes(calib, Mq, R), dtype=torch.uint8, device="cuda")
+    phi = torch.empty((R, wl.N), dtype=torch.float32, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    build_ms = timed(lambda: lukv.lukv_profile_build(calib, U, Mq, ratios, phi, pws), args.steps, max(args.warmup, 3))
+    build_launches = lukv.lukv_last_launch_count()
+
+    p = lukv.make_params(wl.S, wl.L, wl.H, wl.G, wl.d, wl.T, wl.w, wl.kp, wl.dtype, wl.P)
+    q, k, v = synth.gen_tensors(wl, "cuda")
+    ws = lukv.alloc_workspace(p)
+    sigma = np.array([1.0 - wl.keep[i % len(wl.keep)] for i in range(wl.S)], np.float32)
+    budgets = torch.empty((wl.S, wl.N), dtype=torch.int32, device="cuda")
+    offsets = torch.empty((wl.S * wl.N + 1,), dtype=torch.int32, device="cuda")
+    lookup_ms = timed(lambda: lukv.lukv_profile_budgets(p, phi, ratios, sigma, budgets, offsets), 50, 3)
+    rows = int(offsets[-1].item())
+    k_out = torch.empty((rows, wl.d), dtype=k.dtype, device="cuda")
+    v_out = torch.empty((rows, wl.d), dtype=k.dtype, device="cuda")
+    kept = torch.empty((rows,), dtype=torch.int32, device="cuda")
+    scores = torch.empty((wl.S, wl.N, wl.n), dtype=torch.float32, device="cuda")
+    counts = []
+
+    def online():
+        counts.clear()
+        lukv.lukv_profile_budgets(p, phi, ratios, sigma, budgets, offsets)
+        counts.append(lukv.lukv_last_launch_count())
+        lukv.lukv_score(p, q, k, scores, ws)
+        counts.append(lukv.lukv_last_launch_count())
+        lukv.lukv_select_gather(p, scores, budgets, offsets, k, v, k_out, v_out, kept, rows, ws)
+        counts.append(lukv.lukv_last_launch_count())
+
+    sampler = ClockSampler(0)
+    if sampler.ok:
+        sampler.start()
+    online_ms = timed(online, args.steps, max(args.warmup, 3))
+    if sampler.ok and not sampler.samples:
+        sampler.sample_once()
+    sampler.stop()
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import lukv_oracle as O
+        O.build()
+        t0 = time.perf_counter()
+        O.profile_build(U_np[:6], Tc, wl.w, ratios)
+        sec = time.perf_counter() - t0
+        cpu = {"value": 6 * R / sec, "unit": "(query, ratio) allocations/s", "cores": 1, "kind": "oracle",
+               "seconds_for_sample": sec, "sample": f"6 of {Mq} calibration queries, all {R} ratios, single thread"}
+    es = 2 if wl.dtype == "bf16" else 4
+    print(json.dumps({
+        "metric": "offline profile build: (query, ratio) allocations per second", "value": Mq * R / (build_ms * 1e-3),
+        "unit": "(query, ratio) allocations/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": build_ms, "higher_is_better": True, "dtype": "f32 curves / f64 hull and mean / int64 budgets",
+        "data": "synthetic (seeded)", "vs_baseline": None,
+        "config": {"workload": f"profile[{wl.name}]", "queries": Mq, "calibration_tokens": Tc, "heads": wl.N,
+                   "curve_points": Tc + 1, "ratios": R, "curve_bytes": int(U.numel() * 4)},
+        "gpu_launches": build_launches * args.steps,
+        "lookup": {"ms_per_call": lookup_ms, "sequences": wl.S, "heads": wl.N},
+        "online_mode": {"metric": METRIC, "value": wl.S * wl.T / (online_ms * 1e-3), "unit": UNIT,
+                        "ms_per_step": online_ms, "packed_rows": rows, "launches_per_step": sum(counts),
+                        "path_bytes_per_step": wl.S * wl.N * wl.T * wl.d * es + 2 * rows * wl.d * es},
+        "clocks": sampler.summary(), "cpu_baseline": cpu}))
+
+
 def pick_workload(args):
     from paper_2602_08585_b200 import synth
     wl = synth.CONFIGS[args.workload]
@@ -393,6 +488,9 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.path == "profile":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_profile_path(args)
     else:
         run_ours(args)
 
