@@ -253,7 +253,13 @@ struct Plan {
   // + TMA producer, two MMA issuers, helper.  The count stays a multiple of 4 warps: the register
   // file is handed out as if the CTA were rounded up to one.
   static constexpr int kThreads = (kEpiWarps + 4) * 32;
-  static constexpr int kStages = MT == 1 ? 3 : 2;      // key-tile ring
+  // Key-tile ring.  The count must be even: tile t uses stage t % kStages and is issued by issuer
+  // t % 2, so with an even count every stage (its "full" barrier) has one waiting thread.  With an
+  // odd count the two issuers would take turns on a stage, and the one that runs ahead could wait
+  // for a phase two ahead of the barrier -- which a parity wait reports as complete while the
+  // previous load of that stage is still in flight.
+  static constexpr int kStages = MT == 1 ? 4 : 2;
+  static_assert(kStages % 2 == 0, "a key stage must always be consumed by the same MMA issuer");
   static constexpr int kQSlots = 2;                    // query tiles of the job in the tensor pipe and the next one
   static constexpr int kQBytes = MT * kStageBytes;     // [half][MT*128 rows][128 B]
   static constexpr int kFinBufs = 1;                   // blocks of partials in flight while a head is folded
