@@ -20,6 +20,8 @@
 //   select   : top-b positions of a head by the proxy (Sec. 4.3 "Eviction"; M^pi(k) of
 //              Sec. 3.2), ties by lower index (App. A.1 allows any fixed rule).
 //   gather   : the retained index set I of Sec. 3.2 materialised as a packed cache.
+//   deployment settings (App. E): attention sinks always ranked first; a minimum number of
+//              tokens per head handed out before the greedy starts.  Both default to off.
 //   profile  : offline profile = mean over calibration queries of the optimal local ratios
 //              (Sec. 4.3, Eq. "calibration_avg"); online lookup and b = floor((1-r)*n)
 //              (Sec. 4.3 "Online Execution").
@@ -165,12 +167,28 @@ inline int64_t seg_cap(int k, int64_t s, int64_t n) {
 
 struct Item { float gain; int k; int hid; int64_t cap; };
 
+// Tokens of segment k of a head that are still for sale when the head's first f tokens are
+// given to it up front (the minimum retention of App. E).
+inline int64_t seg_cap_after_floor(int k, int64_t s, int64_t n, int64_t f) {
+  const int64_t lo = std::max<int64_t>(static_cast<int64_t>(k) * s, f);
+  const int64_t hi = std::min<int64_t>(static_cast<int64_t>(k + 1) * s, n);
+  return hi > lo ? hi - lo : 0;
+}
+
 // ---- select --------------------------------------------------------------------------
 // First b positions of the order (score descending, index ascending), emitted ascending.
-void select_head(const float* pooled, int n, int b, int32_t* kept) {
+// Attention sinks (App. E: sink size 4): the first n_sink positions rank before every other
+// position whatever their score, so they are kept whenever the budget allows (b >= n_sink)
+// and count towards it.
+void select_head(const float* pooled, int n, int b, int n_sink, int32_t* kept) {
   std::vector<int32_t> order(n);
   std::iota(order.begin(), order.end(), 0);
-  std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t c) { return pooled[a] > pooled[c]; });
+  std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t c) {
+    const bool sa = a < n_sink, sc = c < n_sink;
+    if (sa != sc) return sa;
+    if (sa) return false;  // both sinks: position order (stable)
+    return pooled[a] > pooled[c];
+  });
   std::vector<int32_t> top(order.begin(), order.begin() + b);
   std::sort(top.begin(), top.end());
   std::copy(top.begin(), top.end(), kept);
@@ -235,15 +253,20 @@ void oracle_hull(const float* curves, int N, int P, double* gains_f64, float* ga
 // Items are all (hid,k) with non-zero capacity, ordered by (gain descending, k ascending,
 // hid ascending); they are consumed in that order until B_q tokens are spent, the last
 // one partially.
-int oracle_allocate(const float* curves, int N, int P, int T, int w, int S, const int64_t* budgets_in,
-                    int32_t* budgets, int32_t* offsets) {
-  const int64_t n = T - w, s = T / (P - 1);
+//
+// floor_tokens f (App. E: no head is compressed beyond 99 %, i.e. keeps at least 1 % of its
+// tokens): every head first receives its f highest-ranked tokens, the greedy then spends
+// B_q - N*f on what is left.  f = 0 is the plain greedy.  Returns -1 also when B_q < N*f.
+int oracle_allocate_floor(const float* curves, int N, int P, int T, int w, int S, const int64_t* budgets_in,
+                          int64_t floor_tokens, int32_t* budgets, int32_t* offsets) {
+  const int64_t n = T - w, s = T / (P - 1), f = floor_tokens;
+  if (f < 0 || f > n) return -1;
   std::vector<float> g(static_cast<size_t>(N) * (P - 1));
   oracle_hull(curves, N, P, nullptr, g.data());
   std::vector<Item> items;
   for (int hid = 0; hid < N; ++hid)
     for (int k = 0; k + 1 < P; ++k) {
-      const int64_t cap = seg_cap(k, s, n);
+      const int64_t cap = f == 0 ? seg_cap(k, s, n) : seg_cap_after_floor(k, s, n, f);
       if (cap > 0) items.push_back(Item{g[static_cast<size_t>(hid) * (P - 1) + k], k, hid, cap});
     }
   std::sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
@@ -255,9 +278,9 @@ int oracle_allocate(const float* curves, int N, int P, int T, int w, int S, cons
   offsets[0] = 0;
   for (int q = 0; q < S; ++q) {
     const int64_t B = budgets_in[q];
-    if (B < 0 || B > static_cast<int64_t>(N) * n) return -1;
-    std::vector<int64_t> b(N, 0);
-    int64_t left = B;
+    if (B < static_cast<int64_t>(N) * f || B > static_cast<int64_t>(N) * n) return -1;
+    std::vector<int64_t> b(N, f);
+    int64_t left = B - static_cast<int64_t>(N) * f;
     for (const Item& it : items) {
       if (left == 0) break;
       const int64_t take = std::min(left, it.cap);
@@ -273,6 +296,17 @@ int oracle_allocate(const float* curves, int N, int P, int T, int w, int S, cons
   return 0;
 }
 
+int oracle_allocate(const float* curves, int N, int P, int T, int w, int S, const int64_t* budgets_in,
+                    int32_t* budgets, int32_t* offsets) {
+  return oracle_allocate_floor(curves, N, P, T, w, S, budgets_in, 0, budgets, offsets);
+}
+
+// Tokens every head keeps at least: ceil(min_keep * n), min_keep in [0,1] (App. E uses 0.01).
+int64_t oracle_floor_tokens(float min_keep, int n) {
+  const double f = std::ceil(static_cast<double>(min_keep) * static_cast<double>(n));
+  return f < 0.0 ? 0 : (f > n ? n : static_cast<int64_t>(f));
+}
+
 // Offline profile aggregation (Sec. 4.3 "Profile Aggregation", Eq. "calibration_avg").
 // curves: [Mq][N][P], one set of per-head utility curves per calibration query, taken on a
 // calibration context of T tokens (n = T-w rankable).  ratios: [R] global compression
@@ -280,24 +314,33 @@ int oracle_allocate(const float* curves, int N, int P, int T, int w, int S, cons
 // global budget B(rho) = floor((1-rho)*N*n); the query's optimal local ratio of head hid is
 // r* = 1 - b_hid/n; the profile is the mean of r* over the queries.
 // profile: [R][N], fp64 mean rounded once to fp32.  Returns 0, or -1 for a ratio outside [0,1].
-int oracle_profile_build(const float* curves, int Mq, int N, int P, int T, int w, const float* ratios, int R,
-                         float* profile) {
+// min_keep > 0 (App. E): every head keeps at least f = ceil(min_keep*n) tokens in every solution, and
+// a grid ratio whose budget would fall below N*f is solved for N*f.
+int oracle_profile_build_floor(const float* curves, int Mq, int N, int P, int T, int w, const float* ratios, int R,
+                               float min_keep, float* profile) {
   const int64_t n = T - w;
+  const int64_t f = oracle_floor_tokens(min_keep, static_cast<int>(n));
   std::vector<int64_t> B(R);
   for (int j = 0; j < R; ++j) {
     const double rho = static_cast<double>(ratios[j]);
     if (!(rho >= 0.0 && rho <= 1.0)) return -1;
     B[j] = static_cast<int64_t>(std::floor((1.0 - rho) * static_cast<double>(static_cast<int64_t>(N) * n)));
+    if (B[j] < static_cast<int64_t>(N) * f) B[j] = static_cast<int64_t>(N) * f;
   }
   std::vector<double> acc(static_cast<size_t>(R) * N, 0.0);
   std::vector<int32_t> b(static_cast<size_t>(R) * N), off(static_cast<size_t>(R) * N + 1);
   for (int i = 0; i < Mq; ++i) {
     const float* ci = curves + static_cast<size_t>(i) * N * P;
-    if (oracle_allocate(ci, N, P, T, w, R, B.data(), b.data(), off.data()) != 0) return -1;
+    if (oracle_allocate_floor(ci, N, P, T, w, R, B.data(), f, b.data(), off.data()) != 0) return -1;
     for (size_t e = 0; e < acc.size(); ++e) acc[e] += 1.0 - static_cast<double>(b[e]) / static_cast<double>(n);
   }
   for (size_t e = 0; e < acc.size(); ++e) profile[e] = static_cast<float>(acc[e] / static_cast<double>(Mq));
   return 0;
+}
+
+int oracle_profile_build(const float* curves, int Mq, int N, int P, int T, int w, const float* ratios, int R,
+                         float* profile) {
+  return oracle_profile_build_floor(curves, Mq, N, P, T, w, ratios, R, 0.f, profile);
 }
 
 // Online lookup and budgeting (Sec. 4.3 "Online Execution", steps 1-2).  profile: [R][N] over
@@ -307,9 +350,11 @@ int oracle_profile_build(const float* curves, int Mq, int N, int P, int T, int w
 // itself).  Budgeting: b = floor((1-r)*n) on the n = T-w rankable positions of the new
 // context, all in fp64.  offsets: exclusive scan of (b + w) in head order.
 // Returns 0, or -1 when a sigma lies outside the grid or the grid is not ascending.
-int oracle_profile_budgets(const float* profile, const float* ratios, int R, int N, int T, int w,
-                           const float* sigma, int S, int32_t* budgets, int32_t* offsets) {
+// min_keep > 0: budgets below f = ceil(min_keep*n) are raised to f (App. E).
+int oracle_profile_budgets_floor(const float* profile, const float* ratios, int R, int N, int T, int w,
+                                 const float* sigma, int S, float min_keep, int32_t* budgets, int32_t* offsets) {
   const int64_t n = T - w;
+  const int64_t f = oracle_floor_tokens(min_keep, static_cast<int>(n));
   for (int j = 0; j + 1 < R; ++j)
     if (!(ratios[j] < ratios[j + 1])) return -1;
   int64_t running = 0;
@@ -330,7 +375,8 @@ int oracle_profile_budgets(const float* profile, const float* ratios, int R, int
       double bf = std::floor((1.0 - r) * static_cast<double>(n));
       if (bf < 0.0) bf = 0.0;
       if (bf > static_cast<double>(n)) bf = static_cast<double>(n);
-      const int64_t bq = static_cast<int64_t>(bf);
+      int64_t bq = static_cast<int64_t>(bf);
+      if (bq < f) bq = f;
       budgets[static_cast<size_t>(q) * N + hid] = static_cast<int32_t>(bq);
       running += bq + w;
       offsets[static_cast<size_t>(q) * N + hid + 1] = static_cast<int32_t>(running);
@@ -339,22 +385,30 @@ int oracle_profile_budgets(const float* profile, const float* ratios, int R, int
   return 0;
 }
 
+int oracle_profile_budgets(const float* profile, const float* ratios, int R, int N, int T, int w,
+                           const float* sigma, int S, int32_t* budgets, int32_t* offsets) {
+  return oracle_profile_budgets_floor(profile, ratios, R, N, T, w, sigma, S, 0.f, budgets, offsets);
+}
+
 // Top-b of one head. pooled: [n]; kept: [b], ascending positions.
-void oracle_select(const float* pooled, int n, int b, int32_t* kept) { select_head(pooled, n, b, kept); }
+void oracle_select(const float* pooled, int n, int b, int32_t* kept) { select_head(pooled, n, b, 0, kept); }
+void oracle_select_sink(const float* pooled, int n, int b, int n_sink, int32_t* kept) {
+  select_head(pooled, n, b, n_sink, kept);
+}
 
 // Selection + gather for all heads. scores: [S*N][n]; budgets: [S*N]; offsets: [S*N+1];
 // k,v: [S*N][T][d]; k_out,v_out: [rows][d]; kept_idx: [rows].  For head u the packed rows
 // [off, off+b) hold the kept positions in ascending order and rows [off+b, off+b+w) hold
 // the window positions n..T-1.
-void oracle_select_gather(const float* scores, const int32_t* budgets, const int32_t* offsets, const void* k,
-                          const void* v, int dtype, int heads, int T, int w, int d, void* k_out, void* v_out,
-                          int32_t* kept_idx) {
+void oracle_select_gather_sink(const float* scores, const int32_t* budgets, const int32_t* offsets, const void* k,
+                               const void* v, int dtype, int heads, int T, int w, int d, int n_sink, void* k_out,
+                               void* v_out, int32_t* kept_idx) {
   const int n = T - w;
   const size_t row = static_cast<size_t>(d) * elem_size(dtype);
   for (int64_t u = 0; u < heads; ++u) {
     const int b = budgets[u];
     int32_t* kept = kept_idx + offsets[u];
-    select_head(scores + u * n, n, b, kept);
+    select_head(scores + u * n, n, b, n_sink, kept);
     for (int i = 0; i < w; ++i) kept[b + i] = n + i;
     for (int t = 0; t < b + w; ++t) {
       const size_t src = (static_cast<size_t>(u) * T + kept[t]) * row;
@@ -365,14 +419,22 @@ void oracle_select_gather(const float* scores, const int32_t* budgets, const int
   }
 }
 
+void oracle_select_gather(const float* scores, const int32_t* budgets, const int32_t* offsets, const void* k,
+                          const void* v, int dtype, int heads, int T, int w, int d, void* k_out, void* v_out,
+                          int32_t* kept_idx) {
+  oracle_select_gather_sink(scores, budgets, offsets, k, v, dtype, heads, T, w, d, 0, k_out, v_out, kept_idx);
+}
+
 // The whole path: allocate (hull + greedy) and score are independent; selection needs
 // both; gather follows.  scores_out (may be null): [S*N][n] pooled scores.
-int oracle_compress(const void* q, const void* k, const void* v, const float* curves, const int64_t* budgets_in,
-                    int dtype, int S, int L, int H, int G, int d, int T, int w, int kp, int P, float scale,
-                    void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets, int32_t* offsets,
-                    float* scores_out) {
+// n_sink, min_keep: the deployment settings of App. E (0, 0 switches them off).
+int oracle_compress_ext(const void* q, const void* k, const void* v, const float* curves, const int64_t* budgets_in,
+                        int dtype, int S, int L, int H, int G, int d, int T, int w, int kp, int P, float scale,
+                        int n_sink, float min_keep, void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets,
+                        int32_t* offsets, float* scores_out) {
   const int N = L * H, n = T - w;
-  if (oracle_allocate(curves, N, P, T, w, S, budgets_in, budgets, offsets) != 0) return -1;
+  if (oracle_allocate_floor(curves, N, P, T, w, S, budgets_in, oracle_floor_tokens(min_keep, n), budgets, offsets) != 0)
+    return -1;
   std::vector<float> local;
   float* sc = scores_out;
   if (!sc) {
@@ -380,8 +442,16 @@ int oracle_compress(const void* q, const void* k, const void* v, const float* cu
     sc = local.data();
   }
   oracle_score(q, k, dtype, S, L, H, G, d, T, w, kp, scale, sc);
-  oracle_select_gather(sc, budgets, offsets, k, v, dtype, S * N, T, w, d, k_out, v_out, kept_idx);
+  oracle_select_gather_sink(sc, budgets, offsets, k, v, dtype, S * N, T, w, d, n_sink, k_out, v_out, kept_idx);
   return 0;
+}
+
+int oracle_compress(const void* q, const void* k, const void* v, const float* curves, const int64_t* budgets_in,
+                    int dtype, int S, int L, int H, int G, int d, int T, int w, int kp, int P, float scale,
+                    void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets, int32_t* offsets,
+                    float* scores_out) {
+  return oracle_compress_ext(q, k, v, curves, budgets_in, dtype, S, L, H, G, d, T, w, kp, P, scale, 0, 0.f, k_out, v_out,
+                             kept_idx, budgets, offsets, scores_out);
 }
 
 }  // extern "C"

@@ -40,6 +40,11 @@ def lib() -> ctypes.CDLL:
         _lib.oracle_compress.restype = ctypes.c_int
         _lib.oracle_profile_build.restype = ctypes.c_int
         _lib.oracle_profile_budgets.restype = ctypes.c_int
+        for name in ("oracle_allocate_floor", "oracle_compress_ext", "oracle_profile_build_floor",
+                     "oracle_profile_budgets_floor"):
+            getattr(_lib, name).restype = ctypes.c_int
+        _lib.oracle_floor_tokens.restype = ctypes.c_int64
+        _lib.oracle_floor_tokens.argtypes = [ctypes.c_float, ctypes.c_int]
     return _lib
 
 
@@ -111,28 +116,36 @@ def hull(curves):
     return g64, g32
 
 
-def allocate(curves, T: int, w: int, budgets_in):
-    """curves [N][P], budgets_in [S] -> (budgets int32 [S][N], offsets int32 [S*N+1])."""
+def floor_tokens(min_keep: float, n: int) -> int:
+    """Tokens every head keeps at least (App. E): ceil(min_keep * n)."""
+    return int(lib().oracle_floor_tokens(ctypes.c_float(min_keep), int(n)))
+
+
+def allocate(curves, T: int, w: int, budgets_in, min_keep: float = 0.0):
+    """curves [N][P], budgets_in [S] -> (budgets int32 [S][N], offsets int32 [S*N+1]).
+    min_keep > 0: every head first gets ceil(min_keep*(T-w)) tokens (App. E)."""
     curves = _c(curves, np.float32)
     budgets_in = _c(budgets_in, np.int64)
     N, P = curves.shape
     S = budgets_in.shape[0]
     budgets = np.empty((S, N), np.int32)
     offsets = np.empty(S * N + 1, np.int32)
-    rc = lib().oracle_allocate(_p(curves), N, P, T, w, S, _p(budgets_in), _p(budgets), _p(offsets))
+    f = floor_tokens(min_keep, T - w)
+    rc = lib().oracle_allocate_floor(_p(curves), N, P, T, w, S, _p(budgets_in), ctypes.c_int64(f), _p(budgets),
+                                     _p(offsets))
     if rc != 0:
-        raise ValueError("budget outside [0, N*(T-w)]")
+        raise ValueError("budget outside [N*floor, N*(T-w)]")
     return budgets, offsets
 
 
-def select(pooled, b: int) -> np.ndarray:
+def select(pooled, b: int, n_sink: int = 0) -> np.ndarray:
     pooled = _c(pooled, np.float32)
     kept = np.empty(b, np.int32)
-    lib().oracle_select(_p(pooled), pooled.shape[0], b, _p(kept))
+    lib().oracle_select_sink(_p(pooled), pooled.shape[0], b, int(n_sink), _p(kept))
     return kept
 
 
-def select_gather(scores, budgets, offsets, k, v, w: int):
+def select_gather(scores, budgets, offsets, k, v, w: int, n_sink: int = 0):
     """scores [U][n], budgets [U], offsets [U+1], k/v [U][T][d] -> (k_out, v_out, kept_idx)."""
     scores = _c(scores, np.float32)
     budgets = _c(budgets, np.int32).reshape(-1)
@@ -144,12 +157,13 @@ def select_gather(scores, budgets, offsets, k, v, w: int):
     k_out = np.empty((rows, d), k.dtype)
     v_out = np.empty((rows, d), v.dtype)
     kept = np.empty(rows, np.int32)
-    lib().oracle_select_gather(_p(scores), _p(budgets), _p(offsets), _p(k), _p(v), _dtype_code(k), U, T, w, d,
-                               _p(k_out), _p(v_out), _p(kept))
+    lib().oracle_select_gather_sink(_p(scores), _p(budgets), _p(offsets), _p(k), _p(v), _dtype_code(k), U, T, w, d,
+                                    int(n_sink), _p(k_out), _p(v_out), _p(kept))
     return k_out, v_out, kept
 
 
-def compress(q, k, v, curves, budgets_in, G: int, kp: int, scale: float = 0.0):
+def compress(q, k, v, curves, budgets_in, G: int, kp: int, scale: float = 0.0, n_sink: int = 0,
+             min_keep: float = 0.0):
     """The whole path. Returns dict(k_out, v_out, kept_idx, budgets, offsets, scores)."""
     q, k, v = _c(q), _c(k), _c(v)
     curves = _c(curves, np.float32)
@@ -163,28 +177,30 @@ def compress(q, k, v, curves, budgets_in, G: int, kp: int, scale: float = 0.0):
         k_out=np.empty((rows, d), k.dtype), v_out=np.empty((rows, d), v.dtype),
         kept_idx=np.empty(rows, np.int32), budgets=np.empty((S, N), np.int32),
         offsets=np.empty(S * N + 1, np.int32), scores=np.empty((S, N, T - w), np.float32))
-    rc = lib().oracle_compress(_p(q), _p(k), _p(v), _p(curves), _p(budgets_in), _dtype_code(k), S, L, H, G, d,
-                               T, w, kp, P, ctypes.c_float(scale), _p(out["k_out"]), _p(out["v_out"]),
+    rc = lib().oracle_compress_ext(_p(q), _p(k), _p(v), _p(curves), _p(budgets_in), _dtype_code(k), S, L, H, G, d,
+                               T, w, kp, P, ctypes.c_float(scale), int(n_sink), ctypes.c_float(min_keep),
+                               _p(out["k_out"]), _p(out["v_out"]),
                                _p(out["kept_idx"]), _p(out["budgets"]), _p(out["offsets"]), _p(out["scores"]))
     if rc != 0:
         raise ValueError("budget outside [0, N*(T-w)]")
     return out
 
 
-def profile_build(curves, T: int, w: int, ratios):
+def profile_build(curves, T: int, w: int, ratios, min_keep: float = 0.0):
     """Offline profile (Sec. 4.3, Eq. "calibration_avg"). curves [Mq][N][P] -> profile [R][N] fp32."""
     curves = _c(curves, np.float32)
     ratios = _c(ratios, np.float32)
     Mq, N, P = curves.shape
     R = ratios.shape[0]
     profile = np.empty((R, N), np.float32)
-    rc = lib().oracle_profile_build(_p(curves), Mq, N, P, T, w, _p(ratios), R, _p(profile))
+    rc = lib().oracle_profile_build_floor(_p(curves), Mq, N, P, T, w, _p(ratios), R, ctypes.c_float(min_keep),
+                                          _p(profile))
     if rc != 0:
         raise ValueError("ratio outside [0, 1]")
     return profile
 
 
-def profile_budgets(profile, ratios, T: int, w: int, sigma):
+def profile_budgets(profile, ratios, T: int, w: int, sigma, min_keep: float = 0.0):
     """Online lookup + budgeting (Sec. 4.3). Returns (budgets [S][N] int32, offsets [S*N+1] int32)."""
     profile = _c(profile, np.float32)
     ratios = _c(ratios, np.float32)
@@ -193,7 +209,8 @@ def profile_budgets(profile, ratios, T: int, w: int, sigma):
     S = sigma.shape[0]
     budgets = np.empty((S, N), np.int32)
     offsets = np.empty(S * N + 1, np.int32)
-    rc = lib().oracle_profile_budgets(_p(profile), _p(ratios), R, N, T, w, _p(sigma), S, _p(budgets), _p(offsets))
+    rc = lib().oracle_profile_budgets_floor(_p(profile), _p(ratios), R, N, T, w, _p(sigma), S,
+                                            ctypes.c_float(min_keep), _p(budgets), _p(offsets))
     if rc != 0:
         raise ValueError("sigma outside the ratio grid, or grid not strictly ascending")
     return budgets, offsets
