@@ -71,6 +71,17 @@ typedef struct lukv_params {
   int32_t curve_points; /* P, 2 <= P <= 4097, (P-1) divides T                                 */
   float softmax_scale;  /* 0 selects 1/sqrt(d) (Eq. 1)                                        */
   int32_t flags;        /* reserved, must be 0                                                */
+  /* Deployment settings of App. E (implementation details); 0 switches either off.            */
+  int32_t n_sink;       /* attention sinks: positions 0..n_sink-1 rank before all others in   */
+                        /* the selection whatever their score, so they are kept whenever the  */
+                        /* head's budget allows and count towards it; 0 <= n_sink <= n        */
+                        /* (the paper uses 4)                                                 */
+  float min_keep;       /* minimum retention per head, 0 <= min_keep <= 1 (the paper uses     */
+                        /* 0.01): every head keeps at least f = ceil(min_keep * n) of its n   */
+                        /* rankable tokens (fp64 product of the fp32 value).  Allocation      */
+                        /* hands every head its first f tokens before the greedy spends       */
+                        /* B_q - N*f (B_q < N*f is LUKV_ERR_BUDGET); the profile build        */
+                        /* solves max(B(rho), N*f); the lookup raises budgets below f to f    */
 } lukv_params_t;
 
 /* Bytes of scratch that any of the calls below needs for these parameters (one size fits

@@ -100,9 +100,12 @@ __device__ __forceinline__ unsigned long long seg_key(float gain, unsigned k, un
   return ((unsigned long long)(~__float_as_uint(gain)) << 32) | (unsigned long long)(k * N + hid);
 }
 
-__device__ __forceinline__ long long capsum(int c, int seg, int n) {  // tokens in segments [0,c)
-  const long long t = (long long)c * seg;
-  return t < n ? t : (long long)n;
+// Tokens for sale in segments [0,c) of a head whose first `floor_tok` tokens were handed to it up
+// front (the minimum retention of App. E; 0 = none).
+__device__ __forceinline__ long long capsum(int c, int seg, int n, int floor_tok) {
+  long long t = (long long)c * seg;
+  t = (t < n ? t : (long long)n) - floor_tok;
+  return t > 0 ? t : 0;
 }
 
 // One CTA per sequence.  Within a head the keys increase with k (gains are non-increasing),
@@ -118,7 +121,8 @@ __device__ __forceinline__ long long capsum(int c, int seg, int n) {  // tokens 
 __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __restrict__ gains, GreedyArgs args,
                                                                 int32_t* __restrict__ budgets,
                                                                 int32_t* __restrict__ offsets, SetStride set, int N,
-                                                                int P, int seg, int nseg, int n, int w, int tph) {
+                                                                int P, int seg, int nseg, int n, int w, int tph,
+                                                                int floor_tok) {
   gains += (size_t)blockIdx.y * set.gains;
   budgets += (size_t)blockIdx.y * set.budgets;
   offsets += (size_t)blockIdx.y * set.offsets;
@@ -142,7 +146,7 @@ __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __r
     hi[h] = nseg;
   }
   if (tid == 0) {
-    sh_remaining = args.budget[blockIdx.x];
+    sh_remaining = args.budget[blockIdx.x] - (long long)N * floor_tok;  // the floor is spent before the greedy
     sh_all_taken = 0;
   }
   __syncthreads();
@@ -174,14 +178,16 @@ __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __r
             const unsigned dgt = (unsigned)(seg_key(gv[i], k, h, N) >> shift) & 255u;
             if (dgt != run_digit) {
               if (run_digit != 0xffffffffu)
-                atomicAdd(&hist[run_digit], (unsigned long long)(capsum(k, seg, n) - capsum(run_start, seg, n)));
+                atomicAdd(&hist[run_digit],
+                          (unsigned long long)(capsum(k, seg, n, floor_tok) - capsum(run_start, seg, n, floor_tok)));
               run_start = k;
               run_digit = dgt;
             }
           }
         }
       }
-      atomicAdd(&hist[run_digit], (unsigned long long)(capsum(b, seg, n) - capsum(run_start, seg, n)));
+      atomicAdd(&hist[run_digit],
+                (unsigned long long)(capsum(b, seg, n, floor_tok) - capsum(run_start, seg, n, floor_tok)));
     }
     __syncthreads();
     if (tid < 32) {
@@ -265,7 +271,7 @@ __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __r
   const int h_begin = min(N, tid * per), h_end = min(N, h_begin + per);
   long long local = 0;
   for (int h = h_begin; h < h_end; ++h) {
-    long long b = capsum(lo[h], seg, n);
+    long long b = floor_tok + capsum(lo[h], seg, n, floor_tok);
     if (hi[h] > lo[h]) b += R;  // the one partially bought segment
     lo[h] = (int)b;
     local += b + w;
@@ -331,7 +337,8 @@ cudaError_t launch_greedy(const Dims& dm, const float* gains, const int64_t* bud
     }
     args.seq0 = q0;
     greedy_kernel<<<dim3(cnt, n_sets), kGreedyThreads, greedy_smem, lc.st>>>(gains, args, budgets, offsets, set, dm.N,
-                                                                             dm.P, dm.seg, dm.nseg, dm.n, dm.w, tph);
+                                                                             dm.P, dm.seg, dm.nseg, dm.n, dm.w, tph,
+                                                                             dm.floor_tok);
     lc.mark("greedy");
   }
   return cudaGetLastError();

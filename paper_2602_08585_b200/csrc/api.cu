@@ -45,6 +45,8 @@ static int make_dims(const lukv_params_t* p, Dims* dm) {
       p->window >= p->ctx_len || p->pool_kernel < 1 || p->curve_points < 2)
     return LUKV_ERR_INVALID_ARG;
   if (!(p->softmax_scale >= 0.f) || isinf(p->softmax_scale)) return LUKV_ERR_INVALID_ARG;
+  if (p->n_sink < 0 || p->n_sink > p->ctx_len - p->window || !(p->min_keep >= 0.f) || !(p->min_keep <= 1.f))
+    return LUKV_ERR_INVALID_ARG;
   if (p->head_dim != 64 && p->head_dim != 128) return LUKV_ERR_UNSUPPORTED;
   if (p->dtype != LUKV_DTYPE_BF16 && p->dtype != LUKV_DTYPE_FP32) return LUKV_ERR_UNSUPPORTED;
   if ((p->pool_kernel & 1) == 0) return LUKV_ERR_UNSUPPORTED;
@@ -65,13 +67,16 @@ static int make_dims(const lukv_params_t* p, Dims* dm) {
   dm->nseg = (dm->n + dm->seg - 1) / dm->seg;
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : (float)(1.0 / sqrt((double)dm->d));
   dm->scale_log2 = (float)((double)scale * 1.4426950408889634);
+  dm->n_sink = p->n_sink;
+  const double fl = ceil((double)p->min_keep * (double)dm->n);
+  dm->floor_tok = fl < 0.0 ? 0 : (fl > (double)dm->n ? dm->n : (int)fl);
   return LUKV_OK;
 }
 
 static int check_budgets(const Dims& dm, const int64_t* budgets_in, int64_t* total_rows) {
   int64_t rows = 0;
   for (int q = 0; q < dm.S; ++q) {
-    if (budgets_in[q] < 0 || budgets_in[q] > (int64_t)dm.N * dm.n) return LUKV_ERR_BUDGET;
+    if (budgets_in[q] < (int64_t)dm.N * dm.floor_tok || budgets_in[q] > (int64_t)dm.N * dm.n) return LUKV_ERR_BUDGET;
     rows += budgets_in[q] + (int64_t)dm.N * dm.w;
   }
   *total_rows = rows;
@@ -413,6 +418,7 @@ int lukv_profile_build(const lukv_params_t* calib, const float* curves, int32_t 
       return LUKV_ERR_BUDGET;
     }
     B[j] = (int64_t)floor((1.0 - rho) * (double)((int64_t)dm.N * dm.n));
+    if (B[j] < (int64_t)dm.N * dm.floor_tok) B[j] = (int64_t)dm.N * dm.floor_tok;
   }
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;
@@ -455,7 +461,7 @@ int lukv_profile_budgets(const lukv_params_t* params, const float* profile, cons
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;
   const cudaError_t e =
-      launch_profile_budgets(profile, row_lo, row_hi, frac, dm.S, dm.N, dm.n, dm.w, budgets, offsets, lc);
+      launch_profile_budgets(profile, row_lo, row_hi, frac, dm.S, dm.N, dm.n, dm.w, dm.floor_tok, budgets, offsets, lc);
   free(rows);
   if (e != cudaSuccess) return LUKV_ERR_CUDA;
   g_last_launches = lc.launches;
@@ -467,7 +473,7 @@ const char* lukv_strerror(int code) {
     case LUKV_OK: return "ok";
     case LUKV_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, non-positive size, flags != 0)";
     case LUKV_ERR_UNSUPPORTED: return "unsupported configuration (head_dim, dtype, even pool kernel, curve grid, G*w > 256 or sizes beyond 32 bits)";
-    case LUKV_ERR_BUDGET: return "budget outside [0, N*(T-w)], or a compression ratio outside its range";
+    case LUKV_ERR_BUDGET: return "budget outside [N*ceil(min_keep*(T-w)), N*(T-w)], or a compression ratio outside its range";
     case LUKV_ERR_WORKSPACE_TOO_SMALL: return "workspace smaller than lukv_workspace_bytes()";
     case LUKV_ERR_OUTPUT_TOO_SMALL: return "rows_cap smaller than sum(B_q) + S*N*w";
     case LUKV_ERR_CUDA: return "CUDA launch failed";

@@ -19,6 +19,8 @@ struct Dims {
   int seg;      // tokens per curve segment s = T/(P-1)
   int nseg;     // curve segments with non-zero capacity = ceil(n/seg)
   float scale_log2;  // softmax scale * log2(e): logits are kept in the exp2 domain
+  int n_sink;        // leading positions that rank first in the selection
+  int floor_tok;     // tokens every head keeps at least: ceil(min_keep * n)
   int64_t heads() const { return (int64_t)S * N; }
   size_t esize() const { return dtype == LUKV_DTYPE_BF16 ? 2 : 4; }
 };
@@ -86,7 +88,8 @@ cudaError_t launch_profile_mean(const int32_t* budgets, float* profile, int n_qu
                                 LaunchCtx& lc);
 constexpr int kLookupSeqPerLaunch = 32;
 cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, const int* row_hi, const double* frac,
-                                   int S, int N, int n, int w, int32_t* budgets, int32_t* offsets, LaunchCtx& lc);
+                                   int S, int N, int n, int w, int floor_tok, int32_t* budgets, int32_t* offsets,
+                                   LaunchCtx& lc);
 cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* budgets, const int32_t* offsets,
                           int32_t* kept_idx, int64_t rows_cap, HeadRange hr, LaunchCtx& lc);
 cudaError_t launch_gather(const Dims& dm, const int32_t* offsets, const int32_t* kept_idx, const void* k,

@@ -37,7 +37,7 @@ struct LookupArgs {
 
 // blockIdx.y = sequence of this launch, x covers the heads.
 __global__ void profile_budget_kernel(const float* __restrict__ profile, LookupArgs args, int N, int n,
-                                      int32_t* __restrict__ budgets) {
+                                      int floor_tok, int32_t* __restrict__ budgets) {
   const int hid = blockIdx.x * kProfileThreads + threadIdx.x;
   if (hid >= N) return;
   const int i = blockIdx.y;
@@ -46,7 +46,8 @@ __global__ void profile_budget_kernel(const float* __restrict__ profile, LookupA
   const double r = __dadd_rn(r0, __dmul_rn(__dsub_rn(r1, r0), args.frac[i]));
   double b = floor(__dmul_rn(__dsub_rn(1.0, r), (double)n));
   b = b < 0.0 ? 0.0 : (b > (double)n ? (double)n : b);
-  budgets[(size_t)(args.seq0 + i) * N + hid] = (int32_t)b;
+  const int32_t bi = (int32_t)b;
+  budgets[(size_t)(args.seq0 + i) * N + hid] = bi < floor_tok ? floor_tok : bi;  // minimum retention (App. E)
 }
 
 constexpr int kScanThreads = 1024;
@@ -89,7 +90,8 @@ cudaError_t launch_profile_mean(const int32_t* budgets, float* profile, int n_qu
 }
 
 cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, const int* row_hi, const double* frac,
-                                   int S, int N, int n, int w, int32_t* budgets, int32_t* offsets, LaunchCtx& lc) {
+                                   int S, int N, int n, int w, int floor_tok, int32_t* budgets, int32_t* offsets,
+                                   LaunchCtx& lc) {
   for (int q0 = 0; q0 < S; q0 += kLookupSeqPerLaunch) {
     LookupArgs args;
     const int cnt = S - q0 < kLookupSeqPerLaunch ? S - q0 : kLookupSeqPerLaunch;
@@ -100,7 +102,7 @@ cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, cons
     }
     args.seq0 = q0;
     profile_budget_kernel<<<dim3((N + kProfileThreads - 1) / kProfileThreads, cnt), kProfileThreads, 0, lc.st>>>(
-        profile, args, N, n, budgets);
+        profile, args, N, n, floor_tok, budgets);
     lc.mark("profile_budget");
   }
   offsets_scan_kernel<<<1, kScanThreads, 0, lc.st>>>(budgets, offsets, S * N, w);

@@ -20,6 +20,12 @@ __device__ __forceinline__ uint32_t score_key(float x) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+// Key of position j: attention sinks (the first n_sink positions, App. E) get the largest key, so
+// they rank before every scored position; among themselves the lower position wins like any tie.
+__device__ __forceinline__ uint32_t key_at(const float* src, int j, int n_sink) {
+  return j < n_sink ? 0xFFFFFFFFu : score_key(src[j]);
+}
+
 // Block-wide sum of one int per thread; every thread gets the result.  `buf` is one of
 // two alternating shared arrays so that consecutive calls need a single barrier each.
 __device__ __forceinline__ int block_sum(int v, int* buf) {
@@ -45,7 +51,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
                                                                 const int32_t* __restrict__ budgets,
                                                                 const int32_t* __restrict__ offsets,
                                                                 int32_t* __restrict__ kept_idx, long long rows_cap,
-                                                                int n, int w, int span_rt, int head0) {
+                                                                int n, int w, int span_rt, int head0, int n_sink) {
   __shared__ __align__(16) int cnt_buf[2][kSelWarps];
   __shared__ int scan_gt[kSelWarps], scan_eq[kSelWarps];
   const int u = head0 + blockIdx.x, tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
@@ -68,7 +74,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
 #pragma unroll
     for (int e = 0; e < EPT; ++e) {
       const int j = base + 32 * e;
-      keys[e] = j < n ? score_key(src[j]) : 0u;
+      keys[e] = j < n ? key_at(src, j, n_sink) : 0u;
     }
   }
 
@@ -85,7 +91,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
     } else {
       for (int e = 0; e < iters; ++e) {
         const int j = base + 32 * e;
-        if (j < n) c += score_key(src[j]) >= cand;
+        if (j < n) c += key_at(src, j, n_sink) >= cand;
       }
     }
     if (block_sum(c, cnt_buf[phase]) >= b) thr = cand;
@@ -103,7 +109,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
   } else {
     for (int e = 0; e < iters; ++e) {
       const int j = base + 32 * e;
-      const uint32_t key = j < n ? score_key(src[j]) : 0u;
+      const uint32_t key = j < n ? key_at(src, j, n_sink) : 0u;
       my_gt += key > thr;
       my_eq += key == thr;
     }
@@ -145,7 +151,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
   } else {
     for (int e = 0; e < iters; ++e) {
       const int j = base + 32 * e;
-      emit(j < n ? score_key(src[j]) : 0u, j);
+      emit(j < n ? key_at(src, j, n_sink) : 0u, j);
     }
   }
 }
@@ -234,15 +240,19 @@ cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* bu
   const unsigned grid = (unsigned)hr.nh;
   const int n = dm.n;
   if (n <= kSelThreads * 4)
-    select_kernel<4><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0);
+    select_kernel<4><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
+                                                    dm.n_sink);
   else if (n <= kSelThreads * 16)
-    select_kernel<16><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0);
+    select_kernel<16><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
+                                                    dm.n_sink);
   else if (n <= kSelThreads * 64)
-    select_kernel<64><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0);
+    select_kernel<64><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
+                                                    dm.n_sink);
   else {
     const int per_warp = (n + kSelWarps - 1) / kSelWarps;
     const int span = (per_warp + 31) & ~31;
-    select_kernel<0><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, span, hr.h0);
+    select_kernel<0><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, span, hr.h0,
+                                                   dm.n_sink);
   }
   lc.mark("select");
   return cudaGetLastError();

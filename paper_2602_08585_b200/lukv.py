@@ -30,7 +30,8 @@ class Params(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("n_layers", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("gqa_group", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("ctx_len", ctypes.c_int32),
                 ("window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32), ("dtype", ctypes.c_int32),
-                ("curve_points", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("flags", ctypes.c_int32)]
+                ("curve_points", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("flags", ctypes.c_int32),
+                ("n_sink", ctypes.c_int32), ("min_keep", ctypes.c_float)]
 
     @property
     def N(self):
@@ -89,12 +90,12 @@ def strerror(code: int) -> str:
 
 
 def make_params(S: int, L: int, H: int, G: int, d: int, T: int, w: int, kp: int, dtype, P: int,
-                scale: float = 0.0) -> Params:
+                scale: float = 0.0, n_sink: int = 0, min_keep: float = 0.0) -> Params:
     if isinstance(dtype, torch.dtype):
         dtype = {torch.bfloat16: DTYPE_BF16, torch.float32: DTYPE_FP32}[dtype]
     elif isinstance(dtype, str):
         dtype = {"bf16": DTYPE_BF16, "fp32": DTYPE_FP32}[dtype]
-    return Params(S, L, H, G, d, T, w, kp, int(dtype), P, float(scale), 0)
+    return Params(S, L, H, G, d, T, w, kp, int(dtype), P, float(scale), 0, int(n_sink), float(min_keep))
 
 
 def _ptr(t) -> Optional[int]:

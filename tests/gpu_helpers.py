@@ -61,10 +61,10 @@ def assert_scores_close(gpu: np.ndarray, ref: np.ndarray):
                            f"{(err / np.maximum(np.abs(ref), 1e-300)).max():.3e}")
 
 
-def kept_agreement(kept_gpu, kept_ref, offsets, budgets, scores_ref):
+def kept_agreement(kept_gpu, kept_ref, offsets, budgets, scores_ref, n_sink=0):
     """Fraction of the oracle's kept (non-window) positions that the GPU path kept too; every
     position in the symmetric difference must sit within the score tolerance of the oracle's
-    threshold score of that head."""
+    threshold score of that head (with attention sinks: of its scored, non-sink positions)."""
     budgets = budgets.reshape(-1)
     scores_ref = scores_ref.reshape(budgets.shape[0], -1)
     same = total = 0
@@ -80,7 +80,8 @@ def kept_agreement(kept_gpu, kept_ref, offsets, budgets, scores_ref):
         total += b
         diff = np.setxor1d(g, r, assume_unique=True)
         if len(diff):
-            t = np.sort(scores_ref[u])[::-1][b - 1].astype(np.float64)
+            assert b > n_sink and diff.min() >= n_sink, f"head {u}: a sink position differs"
+            t = np.sort(scores_ref[u][n_sink:])[::-1][b - n_sink - 1].astype(np.float64)
             gap = np.abs(scores_ref[u][diff].astype(np.float64) - t)
             assert np.all(gap <= 2 * (SCORE_RTOL * t + SCORE_ATOL)), f"head {u}: mismatch away from the threshold"
     return same / max(total, 1)

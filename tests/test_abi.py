@@ -121,3 +121,14 @@ def test_profile_argument_errors_come_back_before_any_launch():
     assert lukv.lukv_profile_budgets(p, f, grid, [0.5, 1.25], f, f, check=False) == lukv.ERR_BUDGET
     assert lukv.lukv_profile_budgets(p, f, [0.2, 0.8], [0.1, 0.5], f, f, check=False) == lukv.ERR_BUDGET
     assert lukv.lukv_profile_budgets(p, None, grid, [0.5, 0.5], f, f, check=False) == lukv.ERR_INVALID_ARG
+
+
+def test_deployment_settings_are_validated():
+    f = _Fake()
+    p = _p(min_keep=0.5)                      # n = 248, floor 124 tokens per head, N = 4
+    assert lukv.lukv_allocate(p, f, [4 * 124 - 1], f, f, f, check=False) == lukv.ERR_BUDGET
+    assert lukv.lukv_allocate(_p(min_keep=1.5), f, [10], f, f, f, check=False) == lukv.ERR_INVALID_ARG
+    assert lukv.lukv_allocate(_p(min_keep=-0.1), f, [10], f, f, f, check=False) == lukv.ERR_INVALID_ARG
+    assert lukv.lukv_score(_p(n_sink=-1), f, f, f, f, check=False) == lukv.ERR_INVALID_ARG
+    assert lukv.lukv_score(_p(n_sink=249), f, f, f, f, check=False) == lukv.ERR_INVALID_ARG
+    assert lukv.lukv_workspace_bytes(_p(n_sink=4, min_keep=0.01)) == lukv.lukv_workspace_bytes(_p())
