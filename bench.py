@@ -41,6 +41,10 @@ def parse_args():
     ap.add_argument("--path", default="compress", choices=["compress", "profile"],
                     help="compress: the headline path; profile: the offline profile build and the online "
                          "lookup front end (secondary measurement, single GPU)")
+    ap.add_argument("--sinks", type=int, default=0, help="attention sinks kept in every head (App. E uses 4)")
+    ap.add_argument("--min-keep", type=float, default=0.0,
+                    help="minimum retention per head (App. E uses 0.01); default off, as the headline "
+                         "configuration does not name it")
     ap.add_argument("--layers", type=int, default=0,
                     help="override the workload's layer count (a reduced case for profiler captures)")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -52,7 +56,7 @@ def parse_args():
 
 # ---- CPU oracle leg (cpu_baseline of our arm, and the whole reference arm) --------------------
 
-def oracle_sample_seconds(wl, heads):
+def oracle_sample_seconds(wl, heads, n_sink=0, min_keep=0.0):
     """Seconds the oracle needs for allocation (all heads) plus score/select/gather of `heads`
     sampled heads; returns (seconds, seconds extrapolated to the whole workload)."""
     import numpy as np
@@ -70,14 +74,14 @@ def oracle_sample_seconds(wl, heads):
         qh, kh, vh = synth.gen_head(wl, q, layer, h, "cpu")
         data.append((u, synth.to_numpy_bits(qh), synth.to_numpy_bits(kh), synth.to_numpy_bits(vh)))
     t0 = time.perf_counter()
-    budgets, offsets = O.allocate(curves, wl.T, wl.w, Bs)
+    budgets, offsets = O.allocate(curves, wl.T, wl.w, Bs, min_keep=min_keep)
     t_alloc = time.perf_counter() - t0
     t0 = time.perf_counter()
     for u, qh, kh, vh in data:
         _, pooled = O.score_head(qh, kh, wl.kp)
         b = np.array([budgets.reshape(-1)[u]], np.int32)
         off = np.array([0, b[0] + wl.w], np.int32)
-        O.select_gather(pooled[None], b, off, kh[None], vh[None], wl.w)
+        O.select_gather(pooled[None], b, off, kh[None], vh[None], wl.w, n_sink=n_sink)
     t_heads = time.perf_counter() - t0
     return t_alloc + t_heads, t_alloc + t_heads * total_heads / heads, heads
 
@@ -92,10 +96,10 @@ def run_reference(args):
     wl = pick_workload(args)
     heads = max(1, min(4, wl.S * wl.N))
     for _ in range(args.warmup):
-        oracle_sample_seconds(wl, 1)
+        oracle_sample_seconds(wl, 1, args.sinks, args.min_keep)
     full = []
     for _ in range(args.steps):
-        _, extrap, used = oracle_sample_seconds(wl, heads)
+        _, extrap, used = oracle_sample_seconds(wl, heads, args.sinks, args.min_keep)
         full.append(extrap)
     sec = sum(full) / len(full)
     value = wl.S * wl.T / sec
@@ -103,7 +107,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded)",
-        "config": {"workload": wl.name, "S": wl.S, "heads": wl.N, "T": wl.T, "w": wl.w, "keep": list(wl.keep)},
+        "config": {"workload": wl.name, "S": wl.S, "heads": wl.N, "T": wl.T, "w": wl.w, "keep": list(wl.keep),
+                   "n_sink": args.sinks, "min_keep": args.min_keep},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": f"{heads} of {wl.S * wl.N} heads per step (score+select+gather) plus the full "
                                    "allocation, single thread, extrapolated to all heads"},
@@ -239,7 +244,8 @@ def run_ours(args):
     lukv.lib()
 
     wl = pick_workload(args)
-    p = lukv.make_params(wl.S, wl.L, wl.H, wl.G, wl.d, wl.T, wl.w, wl.kp, wl.dtype, wl.P)
+    p = lukv.make_params(wl.S, wl.L, wl.H, wl.G, wl.d, wl.T, wl.w, wl.kp, wl.dtype, wl.P, n_sink=args.sinks,
+                         min_keep=args.min_keep)
     q, k, v = synth.gen_tensors(wl, "cuda")
     curves_np = synth.gen_curves(wl)
     curves = torch.from_numpy(curves_np).cuda()
@@ -358,7 +364,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import lukv_oracle as O
         O.build()
-        sec, extrap, used = oracle_sample_seconds(wl, args.cpu_heads)
+        sec, extrap, used = oracle_sample_seconds(wl, args.cpu_heads, args.sinks, args.min_keep)
         cpu_baseline = {"value": wl.S * wl.T / extrap, "unit": UNIT, "cores": 1, "kind": "oracle",
                         "seconds_for_sample": sec,
                         "sample": f"{used} of {wl.S * wl.N} heads (score+select+gather) plus the full allocation, "
@@ -372,7 +378,8 @@ def run_ours(args):
             "data": "synthetic (seeded)",
             "config": {"workload": wl.name, "S": wl.S, "layers": wl.L, "kv_heads": wl.H, "gqa_group": wl.G,
                        "head_dim": wl.d, "T": wl.T, "w": wl.w, "pool": wl.kp, "curve_points": wl.P,
-                       "keep": list(wl.keep), "packed_rows": out.rows,
+                       "keep": list(wl.keep), "packed_rows": out.rows, "n_sink": args.sinks,
+                       "min_keep": args.min_keep,
                        "l2": "inputs (K+V %.2f GB) exceed the 126 MB L2; no explicit flush" %
                              (2 * wl.S * wl.N * wl.T * wl.d * es / 1e9),
                        "parallelism": "replicas (one full workload per GPU)" if world > 1 else "single GPU"},
