@@ -74,7 +74,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
 #pragma unroll
     for (int e = 0; e < EPT; ++e) {
       const int j = base + 32 * e;
-      keys[e] = j < n ? key_at(src, j, n_sink) : 0u;
+      keys[e] = j < n ? score_key(src[j]) : 0u;
+    }
+    if (wv * span < n_sink) {  // only the warps whose span starts below n_sink hold sink positions
+#pragma unroll
+      for (int e = 0; e < EPT; ++e)
+        if (base + 32 * e < n_sink) keys[e] = 0xFFFFFFFFu;
     }
   }
 
