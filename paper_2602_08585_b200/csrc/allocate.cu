@@ -2,10 +2,11 @@
 //   hull_kernel    PAVA projection of every head's curve increments onto a non-increasing,
 //                  non-negative sequence (Eq. "marginal_gain"), fp64 with explicit
 //                  round-to-nearest operations, gains rounded once to fp32.
-//   greedy_kernel  the marginal-utility greedy, computed as a weighted radix select: the
-//                  greedy consumes curve segments in the order (gain desc, k asc, hid asc);
-//                  the kernel finds the segment at which the budget runs out and gives
-//                  every head the capacity of its segments before that point.
+//   greedy_kernel  the marginal-utility greedy, computed as a weighted selection: the greedy
+//                  consumes curve segments in the order (gain desc, k asc, hid asc); the
+//                  kernel finds the segment at which the budget runs out by bisection over
+//                  the key bits (one binary search per head and bit) and gives every head
+//                  the capacity of its segments before that point.
 #include "common.cuh"
 
 namespace lukv {
@@ -82,7 +83,7 @@ __global__ void hull_kernel(const float* __restrict__ curves, float* __restrict_
 
 // ---- greedy --------------------------------------------------------------------------
 
-constexpr int kGreedyThreads = 1024;
+constexpr int kGreedyMaxThreads = 1024;
 constexpr int kSeqPerLaunch = 32;
 
 struct GreedyArgs {
@@ -108,172 +109,101 @@ __device__ __forceinline__ long long capsum(int c, int seg, int n, int floor_tok
   return t > 0 ? t : 0;
 }
 
-// One CTA per sequence.  Within a head the keys increase with k (gains are non-increasing),
-// so the segments of a head that still match the key prefix form a range [lo,hi); segments
-// before lo are already bought.  Each of the 8 passes histograms the next key byte of the
-// active segments weighted by capacity, picks the byte at which the remaining budget runs
-// out and narrows every head's range to it.  Keys are unique, so one segment remains: the
-// partially bought one.  `tph` threads (a power of two) share a head and split its range.
+// Block-wide sum; every thread gets the result.  `buf` holds one value per warp; two buffers are
+// used alternately so that one barrier per call is enough.
+__device__ __forceinline__ long long block_sum_ll(long long v, long long* buf) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  if ((threadIdx.x & 31) == 0) buf[threadIdx.x >> 5] = v;
+  __syncthreads();
+  long long total = 0;
+  const int warps = blockDim.x >> 5;
+  for (int x = 0; x < warps; ++x) total += buf[x];
+  return total;
+}
+
+// One CTA per (sequence, curve set), one thread per head (a CTA of fewer threads than heads loops).
+// The greedy buys segments in ascending key order until the budget is spent; the kernel finds the
+// key at which that happens by bisection over the 64 key bits.  Within a head the keys increase
+// with k (gains are non-increasing), so the segments of a head that share the key prefix fixed so
+// far form a range [lo,hi), segments before lo are bought, and inside the range the next key bit is
+// 0 up to some index and 1 from there on: one binary search per head and bit finds that index (no
+// search at all when the range's two ends agree), the capacities below it are summed over the
+// heads, and the budget decides which half holds the cut.  Keys are unique, so after the last bit
+// one segment remains: the partially bought one.
 //
 // blockIdx.y selects one of several independent curve sets (the calibration queries of the
 // offline profile, which share the budgets): set i reads gains + i*set.gains, writes
 // budgets + i*set.budgets and offsets + i*set.offsets.  The hot path launches one set.
-__global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __restrict__ gains, GreedyArgs args,
-                                                                int32_t* __restrict__ budgets,
-                                                                int32_t* __restrict__ offsets, SetStride set, int N,
-                                                                int P, int seg, int nseg, int n, int w, int tph,
-                                                                int floor_tok) {
+__global__ void __launch_bounds__(kGreedyMaxThreads) greedy_kernel(const float* __restrict__ gains, GreedyArgs args,
+                                                                   int32_t* __restrict__ budgets,
+                                                                   int32_t* __restrict__ offsets, SetStride set,
+                                                                   int N, int P, int seg, int nseg, int n, int w,
+                                                                   int floor_tok) {
   gains += (size_t)blockIdx.y * set.gains;
   budgets += (size_t)blockIdx.y * set.budgets;
   offsets += (size_t)blockIdx.y * set.offsets;
   extern __shared__ __align__(16) unsigned char greedy_smem[];
   int* lo = reinterpret_cast<int*>(greedy_smem);  // [N]
   int* hi = lo + N;                               // [N]
-  int* cnt_lt = hi + N;                           // [N] active segments with byte <  chosen byte
-  int* cnt_le = cnt_lt + N;                       // [N] active segments with byte <= chosen byte
-  __shared__ unsigned long long hist[256];
-  __shared__ long long sh_remaining;
-  __shared__ int sh_digit, sh_all_taken;
-  __shared__ long long warp_sums[kGreedyThreads / 32];
+  int* mid = hi + N;                              // [N]
+  __shared__ long long sum_buf[2][kGreedyMaxThreads / 32];
+  __shared__ long long warp_sums[kGreedyMaxThreads / 32];
 
   const int q = args.seq0 + blockIdx.x;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, nthr = blockDim.x;
   const int G1 = P - 1;
-  const int sub = tid & (tph - 1);           // this thread's share of a head
-  const int heads_per_iter = kGreedyThreads / tph;
-  for (int h = tid; h < N; h += kGreedyThreads) {
-    lo[h] = 0;
+  long long R = args.budget[blockIdx.x] - (long long)N * floor_tok;  // the floor is spent before the greedy
+  const bool all_taken = (long long)N * (n - floor_tok) <= R;
+  for (int h = tid; h < N; h += nthr) {
+    lo[h] = all_taken ? nseg : 0;
     hi[h] = nseg;
   }
-  if (tid == 0) {
-    sh_remaining = args.budget[blockIdx.x] - (long long)N * floor_tok;  // the floor is spent before the greedy
-    sh_all_taken = 0;
-  }
-  __syncthreads();
-
-  for (int pass = 0; pass < 8; ++pass) {
-    const int shift = 56 - 8 * pass;
-    if (tid < 256) hist[tid] = 0ull;
-    for (int h = tid; h < N; h += kGreedyThreads) {
-      cnt_lt[h] = 0;
-      cnt_le[h] = 0;
-    }
-    __syncthreads();
-    for (int h = tid / tph; h < N; h += heads_per_iter) {
-      const int l = lo[h], r = hi[h];
-      const int len = r - l;
-      const int a = l + (int)(((long long)len * sub) / tph), b = l + (int)(((long long)len * (sub + 1)) / tph);
-      if (a >= b) continue;
-      const float* g = gains + (size_t)h * G1;
-      int run_start = a;
-      unsigned run_digit = 0xffffffffu;
-      for (int k0 = a; k0 < b; k0 += 8) {
-        float gv[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) gv[i] = (k0 + i < b) ? __ldg(g + k0 + i) : 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int k = k0 + i;
-          if (k < b) {
-            const unsigned dgt = (unsigned)(seg_key(gv[i], k, h, N) >> shift) & 255u;
-            if (dgt != run_digit) {
-              if (run_digit != 0xffffffffu)
-                atomicAdd(&hist[run_digit],
-                          (unsigned long long)(capsum(k, seg, n, floor_tok) - capsum(run_start, seg, n, floor_tok)));
-              run_start = k;
-              run_digit = dgt;
+  // (each thread only ever touches the heads it owns, so lo/hi/mid need no barrier of their own)
+  if (!all_taken) {
+    for (int bit = 63; bit >= 0; --bit) {
+      long long local = 0;
+      for (int h = tid; h < N; h += nthr) {
+        const int l = lo[h], r = hi[h];
+        int m = l;
+        if (l < r) {
+          const float* g = gains + (size_t)h * G1;
+          auto bit_at = [&](int k) { return (int)((seg_key(__ldg(g + k), k, h, N) >> bit) & 1ull); };
+          if (bit_at(l)) {
+            m = l;
+          } else if (!bit_at(r - 1)) {
+            m = r;
+          } else {
+            int a = l, b = r - 1;  // bit(a) == 0, bit(b) == 1
+            while (b - a > 1) {
+              const int c = (a + b) >> 1;
+              if (bit_at(c)) b = c; else a = c;
             }
+            m = b;
           }
         }
+        mid[h] = m;
+        local += capsum(m, seg, n, floor_tok) - capsum(l, seg, n, floor_tok);
       }
-      atomicAdd(&hist[run_digit],
-                (unsigned long long)(capsum(b, seg, n, floor_tok) - capsum(run_start, seg, n, floor_tok)));
-    }
-    __syncthreads();
-    if (tid < 32) {
-      // lane owns bins [8*lane, 8*lane+8); find the first bin whose running total exceeds
-      // the remaining budget
-      const long long R = sh_remaining;
-      long long mine = 0;
-#pragma unroll
-      for (int b = 0; b < 8; ++b) mine += (long long)hist[tid * 8 + b];
-      long long incl = mine;
-#pragma unroll
-      for (int off = 1; off < 32; off <<= 1) {
-        const long long o = __shfl_up_sync(0xffffffffu, incl, off);
-        if (tid >= off) incl += o;
-      }
-      const long long excl = incl - mine;
-      const long long total = __shfl_sync(0xffffffffu, incl, 31);
-      if (total <= R) {
-        if (tid == 0) {
-          sh_all_taken = 1;
-          sh_remaining = R - total;
-        }
-      } else if (excl <= R && R < incl) {
-        long long run = excl;
-        for (int b = 0; b < 8; ++b) {
-          const long long hval = (long long)hist[tid * 8 + b];
-          if (run + hval > R) {
-            sh_digit = tid * 8 + b;
-            sh_remaining = R - run;
-            break;
-          }
-          run += hval;
-        }
+      const long long tokens0 = block_sum_ll(local, sum_buf[bit & 1]);
+      if (tokens0 > R) {
+        for (int h = tid; h < N; h += nthr) hi[h] = mid[h];
+      } else {
+        R -= tokens0;
+        for (int h = tid; h < N; h += nthr) lo[h] = mid[h];
       }
     }
-    __syncthreads();
-    if (sh_all_taken) {
-      for (int h = tid; h < N; h += kGreedyThreads) lo[h] = hi[h];
-      break;
-    }
-    // bytes are non-decreasing in k, so counting the active segments below / up to the chosen
-    // byte gives the narrowed range
-    const unsigned D = (unsigned)sh_digit;
-    for (int h = tid / tph; h < N; h += heads_per_iter) {
-      const int l = lo[h], r = hi[h];
-      const int len = r - l;
-      const int a = l + (int)(((long long)len * sub) / tph), b = l + (int)(((long long)len * (sub + 1)) / tph);
-      if (a >= b) continue;
-      const float* g = gains + (size_t)h * G1;
-      int lt = 0, le = 0;
-      for (int k0 = a; k0 < b; k0 += 8) {
-        float gv[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) gv[i] = (k0 + i < b) ? __ldg(g + k0 + i) : 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int k = k0 + i;
-          if (k < b) {
-            const unsigned dgt = (unsigned)(seg_key(gv[i], k, h, N) >> shift) & 255u;
-            lt += dgt < D;
-            le += dgt <= D;
-          }
-        }
-      }
-      if (lt) atomicAdd(&cnt_lt[h], lt);
-      if (le) atomicAdd(&cnt_le[h], le);
-    }
-    __syncthreads();
-    for (int h = tid; h < N; h += kGreedyThreads) {
-      const int l = lo[h];
-      lo[h] = l + cnt_lt[h];
-      hi[h] = l + cnt_le[h];
-    }
-    __syncthreads();
   }
-  __syncthreads();
 
   // budgets, then offsets = row_base + exclusive scan of (budget + w)
-  const long long R = sh_remaining;
-  const int per = (N + kGreedyThreads - 1) / kGreedyThreads;
+  const int per = (N + nthr - 1) / nthr;
   const int h_begin = min(N, tid * per), h_end = min(N, h_begin + per);
+  __syncthreads();  // the scan below re-partitions the heads over the threads
   long long local = 0;
   for (int h = h_begin; h < h_end; ++h) {
     long long b = floor_tok + capsum(lo[h], seg, n, floor_tok);
     if (hi[h] > lo[h]) b += R;  // the one partially bought segment
-    lo[h] = (int)b;
+    mid[h] = (int)b;
     local += b + w;
   }
   long long incl = local;
@@ -289,8 +219,8 @@ __global__ void __launch_bounds__(kGreedyThreads) greedy_kernel(const float* __r
   long long run = args.row_base[blockIdx.x] + before + incl - local;
   if (q == 0 && tid == 0) offsets[0] = 0;
   for (int h = h_begin; h < h_end; ++h) {
-    budgets[(size_t)q * N + h] = lo[h];
-    run += lo[h] + w;
+    budgets[(size_t)q * N + h] = mid[h];
+    run += mid[h] + w;
     offsets[(size_t)q * N + h + 1] = (int32_t)run;
   }
 }
@@ -313,9 +243,9 @@ cudaError_t launch_hull(const float* curves, float* gains, int64_t n_curves, int
 cudaError_t launch_greedy(const Dims& dm, const float* gains, const int64_t* budgets_host, int32_t* budgets,
                           int32_t* offsets, int n_sets, LaunchCtx& lc) {
   cudaError_t e;
-  const size_t greedy_smem = (size_t)dm.N * 4 * sizeof(int);
-  int tph = 1;  // threads per head: the largest power of two <= 1024/N, at most 32
-  while (tph < 32 && tph * 2 * dm.N <= kGreedyThreads) tph *= 2;
+  const size_t greedy_smem = (size_t)dm.N * 3 * sizeof(int);
+  int threads = (dm.N + 31) & ~31;  // one thread per head, whole warps
+  if (threads > kGreedyMaxThreads) threads = kGreedyMaxThreads;
   if ((e = cudaFuncSetAttribute(greedy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)greedy_smem)) != cudaSuccess)
     return e;
   SetStride set;
@@ -336,9 +266,8 @@ cudaError_t launch_greedy(const Dims& dm, const float* gains, const int64_t* bud
       base += budgets_host[q0 + i] + (long long)dm.N * dm.w;
     }
     args.seq0 = q0;
-    greedy_kernel<<<dim3(cnt, n_sets), kGreedyThreads, greedy_smem, lc.st>>>(gains, args, budgets, offsets, set, dm.N,
-                                                                             dm.P, dm.seg, dm.nseg, dm.n, dm.w, tph,
-                                                                             dm.floor_tok);
+    greedy_kernel<<<dim3(cnt, n_sets), threads, greedy_smem, lc.st>>>(gains, args, budgets, offsets, set, dm.N, dm.P,
+                                                                      dm.seg, dm.nseg, dm.n, dm.w, dm.floor_tok);
     lc.mark("greedy");
   }
   return cudaGetLastError();
