@@ -1,7 +1,8 @@
 // Stage (b): global head-level budget allocation (paper Sec. 4.2, App. A.2).
 //   hull_kernel    PAVA projection of every head's curve increments onto a non-increasing,
-//                  non-negative sequence (Eq. "marginal_gain"), fp64 with explicit
-//                  round-to-nearest operations, gains rounded once to fp32.
+//                  non-negative sequence (Eq. "marginal_gain"); merge decisions equal to the
+//                  comparison of fp64 block means, gains fp64 with explicit round-to-nearest
+//                  operations, rounded once to fp32.
 //   greedy_kernel  the marginal-utility greedy, computed as a weighted selection: the greedy
 //                  consumes curve segments in the order (gain desc, k asc, hid asc); the
 //                  kernel finds the segment at which the budget runs out by bisection over
@@ -14,20 +15,22 @@ namespace {
 
 // ---- hull ----------------------------------------------------------------------------
 
-// mean of block [l1,r1) <= mean of block [l2,r2), where the mean of [l,r) is (U[r]-U[l])/(r-l),
-// decided exactly as the comparison of the two correctly rounded fp64 quotients.  Three tiers,
-// cheapest first (the fp64 pipe is slow, and the walk below is one dependent chain):
+// mean of block 1 <= mean of block 2, where a block's mean is (its curve rise) / (its length) and
+// the rises are differences of two fp32 curve values: decided exactly as the comparison of the two
+// correctly rounded fp64 quotients.  Three tiers, cheapest first (the fp64 pipe is slow, and the
+// walk below is one dependent chain):
 //   fp32 cross products, when they are further apart than fp32 rounding can explain;
 //   fp64 cross products, when they are clearly apart;
 //   the fp64 quotients themselves.
-__device__ __forceinline__ bool mean_le(const float* U, int l1, int r1, int l2, int r2) {
-  const float fa = U[r1] - U[l1], fb = (float)(r1 - l1), fc = U[r2] - U[l2], fd = (float)(r2 - l2);
+// Block 1 rises from u_l1 to u_r1 over len1 points, block 2 from u_l2 to u_r2 over len2.
+__device__ __forceinline__ bool mean_le(float u_l1, float u_r1, int len1, float u_l2, float u_r2, int len2) {
+  const float fa = u_r1 - u_l1, fb = (float)len1, fc = u_r2 - u_l2, fd = (float)len2;
   const float q1 = fa * fd, q2 = fc * fb;
   const float ftol = 4e-7f * fmaxf(fabsf(q1), fabsf(q2));  // each product carries two roundings of 2^-24
   if (q1 < q2 - ftol) return true;
   if (q1 > q2 + ftol) return false;
-  const double a = __dsub_rn((double)U[r1], (double)U[l1]), b = (double)(r1 - l1);
-  const double c = __dsub_rn((double)U[r2], (double)U[l2]), d = (double)(r2 - l2);
+  const double a = __dsub_rn((double)u_r1, (double)u_l1), b = (double)len1;
+  const double c = __dsub_rn((double)u_r2, (double)u_l2), d = (double)len2;
   const double p1 = __dmul_rn(a, d), p2 = __dmul_rn(c, b);
   const double diff = __dsub_rn(p1, p2);
   const double tol = fmax(fabs(p1), fabs(p2)) * 9.094947017729282e-13;  // 2^-40
@@ -36,12 +39,17 @@ __device__ __forceinline__ bool mean_le(const float* U, int l1, int r1, int l2, 
   return __ddiv_rn(a, b) <= __ddiv_rn(c, d);
 }
 
-// Shared memory of one warp of the hull kernel: [P] floats, [P] ints, [P] floats.
-__host__ __device__ inline size_t hull_bytes_per_warp(int P) { return ((size_t)P * 12 + 15) & ~(size_t)15; }
+// Shared memory of one warp of the hull kernel: the stack of block starts, [P] 16-bit indices.
+__host__ __device__ inline size_t hull_bytes_per_warp(int P) { return ((size_t)P * 2 + 15) & ~(size_t)15; }
 
-// One warp per head.  Lane 0 runs the pool-adjacent-violators stack (the sequence of merge
-// decisions is the algorithm; it is serial by nature) with the top block cached in registers;
-// the other lanes stage the curve into shared memory and write the gains out.
+// One warp per curve.  Lane 0 runs the pool-adjacent-violators stack (the sequence of merge
+// decisions is the algorithm; it is serial by nature).  The walk is one dependent chain, so what it
+// touches per step is kept short: the curve values at the starts of the top block and of the
+// current block live in registers, the next curve point is requested one step ahead (the curve is
+// read through L1: the walk streams it, a pop re-reads a point that was read not long before), and
+// the stack of block starts is the only thing in shared memory (2 bytes per point, so that many
+// warps fit an SM when thousands of long curves are projected at once).  The other lanes join for
+// the output: one block of the result per lane at a time.
 // Stack entries are block start points; a block's end is the next entry's start.
 __global__ void hull_kernel(const float* __restrict__ curves, float* __restrict__ gains, int N, int P) {
   extern __shared__ __align__(16) unsigned char hull_smem[];
@@ -49,36 +57,43 @@ __global__ void hull_kernel(const float* __restrict__ curves, float* __restrict_
   const int warps = blockDim.x >> 5;
   const int hid = blockIdx.x * warps + warp;
   if (hid >= N) return;  // whole warps leave together; only __syncwarp is used below
-  float* Us = reinterpret_cast<float*>(hull_smem + (size_t)warp * hull_bytes_per_warp(P));  // [P] curve
-  int* Ls = reinterpret_cast<int*>(Us + P);                                                  // [P] stack of block starts
-  float* Gs = Us + 2 * P;                                                                     // [P-1] gains
-  for (int p = lane; p < P; p += 32) Us[p] = curves[(size_t)hid * P + p];
-  __syncwarp();
+  const float* U = curves + (size_t)hid * P;
+  unsigned short* Ls = reinterpret_cast<unsigned short*>(hull_smem + (size_t)warp * hull_bytes_per_warp(P));
   int sp = 0;
   if (lane == 0) {
-    int top_l = 0;  // start of the block on top of the stack; it ends where the current block starts
+    int top_l = 0;        // start of the block on top of the stack; it ends where the current block starts
+    float u_top = 0.f;    // U[top_l]
+    float u_k = __ldg(U), u_next = __ldg(U + 1);
     for (int k = 0; k + 1 < P; ++k) {
+      const float u_ahead = k + 2 < P ? __ldg(U + k + 2) : 0.f;  // for the next step
       int cur_l = k;
-      while (sp > 0 && mean_le(Us, top_l, cur_l, cur_l, k + 1)) {
+      float u_cur = u_k;  // U[cur_l]
+      while (sp > 0 && mean_le(u_top, u_cur, cur_l - top_l, u_cur, u_next, k + 1 - cur_l)) {
         cur_l = top_l;
+        u_cur = u_top;
         --sp;
-        if (sp > 0) top_l = Ls[sp - 1];
+        if (sp > 0) {
+          top_l = Ls[sp - 1];
+          u_top = __ldg(U + top_l);
+        }
       }
-      Ls[sp++] = cur_l;
+      Ls[sp++] = (unsigned short)cur_l;
       top_l = cur_l;
+      u_top = u_cur;
+      u_k = u_next;
+      u_next = u_ahead;
     }
   }
   sp = __shfl_sync(0xffffffffu, sp, 0);
   __syncwarp();
+  float* out = gains + (size_t)hid * (P - 1);
   for (int i = lane; i < sp; i += 32) {
     const int l = Ls[i];
-    const int r = (i + 1 < sp) ? Ls[i + 1] : P - 1;
-    const double mean = __ddiv_rn(__dsub_rn((double)Us[r], (double)Us[l]), (double)(r - l));
+    const int r = (i + 1 < sp) ? (int)Ls[i + 1] : P - 1;
+    const double mean = __ddiv_rn(__dsub_rn((double)__ldg(U + r), (double)__ldg(U + l)), (double)(r - l));
     const float g = __double2float_rn(mean > 0.0 ? mean : 0.0);
-    for (int k = l; k < r; ++k) Gs[k] = g;
+    for (int k = l; k < r; ++k) out[k] = g;
   }
-  __syncwarp();
-  for (int k = lane; k + 1 < P; k += 32) gains[(size_t)hid * (P - 1) + k] = Gs[k];
 }
 
 // ---- greedy --------------------------------------------------------------------------
@@ -228,9 +243,12 @@ __global__ void __launch_bounds__(kGreedyMaxThreads) greedy_kernel(const float* 
 }  // namespace
 
 cudaError_t launch_hull(const float* curves, float* gains, int64_t n_curves, int P, LaunchCtx& lc) {
-  // one warp per curve, up to 4 warps per block (12 bytes of shared memory per curve point and warp)
-  int hw = (int)((200u * 1024u) / hull_bytes_per_warp(P));
-  hw = hw > 4 ? 4 : (hw < 1 ? 1 : hw);
+  // one warp per curve; few curves: small blocks, so that they spread over the SMs (each walk is a
+  // latency-bound chain); many curves: up to 8 warps per block
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  int hw = (int)((n_curves + sms - 1) / sms);
+  hw = hw > 8 ? 8 : (hw < 1 ? 1 : hw);
   const size_t hull_smem = hull_bytes_per_warp(P) * hw;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(hull_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hull_smem)) != cudaSuccess)
