@@ -26,21 +26,6 @@ __device__ __forceinline__ uint32_t key_at(const float* src, int j, int n_sink) 
   return j < n_sink ? 0xFFFFFFFFu : score_key(src[j]);
 }
 
-// Block-wide sum of one int per thread; every thread gets the result.  `buf` is one of
-// two alternating shared arrays so that consecutive calls need a single barrier each.
-__device__ __forceinline__ int block_sum(int v, int* buf) {
-  v = __reduce_add_sync(0xffffffffu, v);
-  if ((threadIdx.x & 31) == 0) buf[threadIdx.x >> 5] = v;
-  __syncthreads();
-  int total = 0;
-#pragma unroll
-  for (int i = 0; i < kSelWarps; i += 4) {
-    const int4 t = *reinterpret_cast<const int4*>(buf + i);
-    total += t.x + t.y + t.z + t.w;
-  }
-  return total;
-}
-
 // One CTA per head.  Warp wv owns the positions [wv*span, (wv+1)*span) and lane l of it the
 // positions wv*span + e*32 + l, so loads are coalesced and position order is (warp, e, lane).
 // EPT > 0: span = 32*EPT and the thread keeps its EPT keys in registers (n <= 512*EPT).
@@ -52,8 +37,9 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
                                                                 const int32_t* __restrict__ offsets,
                                                                 int32_t* __restrict__ kept_idx, long long rows_cap,
                                                                 int n, int w, int span_rt, int head0, int n_sink) {
-  __shared__ __align__(16) int cnt_buf[2][kSelWarps];
+  __shared__ int hist[2048];
   __shared__ int scan_gt[kSelWarps], scan_eq[kSelWarps];
+  __shared__ int sel_digit, sel_want;
   const int u = head0 + blockIdx.x, tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
   const int b = budgets[u];
   const long long off = offsets[u];
@@ -83,24 +69,65 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
     }
   }
 
-  // b-th largest key: largest thr with count(key >= thr) >= b.  Positions beyond n carry
-  // key 0 and are never counted because every candidate is non-zero.
+  // b-th largest key: the largest thr with count(key >= thr) >= b, found digit by digit (11, 11 and
+  // 10 bits, most significant first): the keys that match the digits fixed so far are counted into
+  // a shared-memory histogram of the next digit, and the bin in which the count of larger keys
+  // reaches the remaining budget is the next digit of thr.  Positions beyond n take no part.
   uint32_t thr = 0;
-  int phase = 0;
-  for (int bit = 31; bit >= 0; --bit) {
-    const uint32_t cand = thr | (1u << bit);
-    int c = 0;
-    if (EPT > 0) {
+  {
+    int want = b;  // keys still to be found among those that match the fixed digits
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+      const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+      const int bins = pass == 2 ? 1024 : 2048;
+      const uint32_t above = pass == 0 ? 0u : (thr >> (shift + (pass == 1 ? 11 : 10)));  // the fixed digits
+      for (int i = tid; i < bins; i += kSelThreads) hist[i] = 0;
+      __syncthreads();
+      auto count = [&](uint32_t key, int j) {
+        if (j < n && (pass == 0 || (key >> (shift + (pass == 1 ? 11 : 10))) == above))
+          atomicAdd(&hist[(key >> shift) & (uint32_t)(bins - 1)], 1);
+      };
+      if (EPT > 0) {
 #pragma unroll
-      for (int e = 0; e < EPT; ++e) c += keys[e] >= cand;
-    } else {
-      for (int e = 0; e < iters; ++e) {
-        const int j = base + 32 * e;
-        if (j < n) c += key_at(src, j, n_sink) >= cand;
+        for (int e = 0; e < EPT; ++e) count(keys[e], base + 32 * e);
+      } else {
+        for (int e = 0; e < iters; ++e) {
+          const int j = base + 32 * e;
+          count(j < n ? key_at(src, j, n_sink) : 0u, j);
+        }
       }
+      __syncthreads();
+      // thread t owns the bins [t*per, t*per+per); suffix sums over the threads, from the top
+      const int per = bins / kSelThreads;  // 4 or 2
+      int mine = 0;
+      for (int i = 0; i < per; ++i) mine += hist[tid * per + i];
+      int incl = mine;  // sum over the lanes >= this one
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += o;
+      }
+      if (lane == 0) scan_gt[wv] = incl;  // warp totals (scan_gt is free until the emit phase)
+      __syncthreads();
+      int higher = 0;  // keys in bins above this thread's bins
+      for (int x = wv + 1; x < kSelWarps; ++x) higher += scan_gt[x];
+      higher += incl - mine;
+      if (higher < want && want <= higher + mine) {  // exactly one thread: the digit is in its bins
+        int run = higher;
+        for (int i = per - 1; i >= 0; --i) {
+          const int c = hist[tid * per + i];
+          if (want <= run + c) {
+            sel_digit = tid * per + i;
+            sel_want = want - run;
+            break;
+          }
+          run += c;
+        }
+      }
+      __syncthreads();
+      thr |= (uint32_t)sel_digit << shift;
+      want = sel_want;
     }
-    if (block_sum(c, cnt_buf[phase]) >= b) thr = cand;
-    phase ^= 1;
   }
 
   // per-warp totals of keys above / equal to the threshold, then an exclusive scan over warps
