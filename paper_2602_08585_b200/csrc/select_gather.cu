@@ -11,7 +11,7 @@
 namespace lukv {
 namespace {
 
-constexpr int kSelThreads = 512;
+constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
 
 // Order-preserving map float -> uint32 (larger float <=> larger key).
@@ -28,7 +28,7 @@ __device__ __forceinline__ uint32_t key_at(const float* src, int j, int n_sink) 
 
 // One CTA per head.  Warp wv owns the positions [wv*span, (wv+1)*span) and lane l of it the
 // positions wv*span + e*32 + l, so loads are coalesced and position order is (warp, e, lane).
-// EPT > 0: span = 32*EPT and the thread keeps its EPT keys in registers (n <= 512*EPT).
+// EPT > 0: span = 32*EPT and the thread keeps its EPT keys in registers (n <= 1024*EPT).
 // EPT == 0: span is a multiple of 32 given by the host and the keys are re-read from memory
 // in every round (long contexts).
 template <int EPT>
@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
       }
       __syncthreads();
       // thread t owns the bins [t*per, t*per+per); suffix sums over the threads, from the top
-      const int per = bins / kSelThreads;  // 4 or 2
+      const int per = bins / kSelThreads;  // 2 or 1
       int mine = 0;
       for (int i = 0; i < per; ++i) mine += hist[tid * per + i];
       int incl = mine;  // sum over the lanes >= this one
@@ -271,14 +271,14 @@ cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* bu
   cudaStream_t st = lc.st;
   const unsigned grid = (unsigned)hr.nh;
   const int n = dm.n;
-  if (n <= kSelThreads * 4)
-    select_kernel<4><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
+  if (n <= kSelThreads * 2)
+    select_kernel<2><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
                                                     dm.n_sink);
-  else if (n <= kSelThreads * 16)
-    select_kernel<16><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
+  else if (n <= kSelThreads * 8)
+    select_kernel<8><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
                                                     dm.n_sink);
-  else if (n <= kSelThreads * 64)
-    select_kernel<64><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
+  else if (n <= kSelThreads * 32)
+    select_kernel<32><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
                                                     dm.n_sink);
   else {
     const int per_warp = (n + kSelWarps - 1) / kSelWarps;
