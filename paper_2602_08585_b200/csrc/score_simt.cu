@@ -209,6 +209,33 @@ __global__ void max_pool_kernel(const float* __restrict__ raw, float* __restrict
   pooled[(size_t)u * n + j] = best;
 }
 
+// The same pooling, four outputs per thread with 16-byte accesses, for rows whose length is a multiple
+// of four (then every row starts on a 16-byte boundary) and windows of at most nine positions: the
+// outputs 4t..4t+3 need the inputs 4t-4..4t+7, three aligned vectors.  Positions outside [0,n) count
+// as -inf (the window is clipped at the ends).
+__global__ void max_pool4_kernel(const float4* __restrict__ raw, float4* __restrict__ pooled, int n4, int half,
+                                 int tiles, int head0) {
+  const int u = head0 + blockIdx.x / tiles;
+  const int t = (blockIdx.x % tiles) * blockDim.x + threadIdx.x;
+  if (t >= n4) return;
+  const float4* r = raw + (size_t)u * n4;
+  const float ninf = -INFINITY;
+  const float4 a = t > 0 ? r[t - 1] : make_float4(ninf, ninf, ninf, ninf);
+  const float4 b = r[t];
+  const float4 c = t + 1 < n4 ? r[t + 1] : make_float4(ninf, ninf, ninf, ninf);
+  const float x[12] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w, c.x, c.y, c.z, c.w};
+  float y[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float best = x[4 + i];
+#pragma unroll
+    for (int d = 1; d <= 4; ++d)
+      if (d <= half) best = fmaxf(best, fmaxf(x[4 + i - d], x[4 + i + d]));
+    y[i] = best;
+  }
+  pooled[(size_t)u * n4 + t] = make_float4(y[0], y[1], y[2], y[3]);
+}
+
 template <typename TIn, int D, int RPT>
 cudaError_t launch_sweeps(const Dims& dm, const void* q, const void* k, const Workspace& ws, LaunchCtx& lc) {
   cudaStream_t st = lc.st;
@@ -261,8 +288,17 @@ cudaError_t launch_lse(const Dims& dm, const float* stats, float* lse, int chunk
 }
 
 cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, HeadRange hr, LaunchCtx& lc) {
-  const int tiles = (dm.n + 255) / 256;
-  max_pool_kernel<<<(unsigned)((int64_t)hr.nh * tiles), 256, 0, lc.st>>>(raw, pooled, dm.n, dm.kp / 2, tiles, hr.h0);
+  const int half = dm.kp / 2;
+  const bool vec = dm.n % 4 == 0 && half <= 4 && (reinterpret_cast<uintptr_t>(raw) & 15u) == 0 &&
+                   (reinterpret_cast<uintptr_t>(pooled) & 15u) == 0;
+  if (vec) {
+    const int n4 = dm.n / 4, tiles = (n4 + 255) / 256;
+    max_pool4_kernel<<<(unsigned)((int64_t)hr.nh * tiles), 256, 0, lc.st>>>(
+        reinterpret_cast<const float4*>(raw), reinterpret_cast<float4*>(pooled), n4, half, tiles, hr.h0);
+  } else {
+    const int tiles = (dm.n + 255) / 256;
+    max_pool_kernel<<<(unsigned)((int64_t)hr.nh * tiles), 256, 0, lc.st>>>(raw, pooled, dm.n, half, tiles, hr.h0);
+  }
   lc.mark("max_pool");
   return cudaGetLastError();
 }
