@@ -20,6 +20,8 @@
 //   select   : top-b positions of a head by the proxy (Sec. 4.3 "Eviction"; M^pi(k) of
 //              Sec. 3.2), ties by lower index (App. A.1 allows any fixed rule).
 //   gather   : the retained index set I of Sec. 3.2 materialised as a packed cache.
+//   curves   : utility-versus-budget curve of a proxy metric = running sum of the oracle
+//              importance in the metric's ranking order (Sec. 3.2, Eq. "head_loss_def").
 //   deployment settings (App. E): attention sinks always ranked first; a minimum number of
 //              tokens per head handed out before the greedy starts.  Both default to off.
 //   profile  : offline profile = mean over calibration queries of the optimal local ratios
@@ -33,7 +35,8 @@
 // uniform budgets against a library-op SnapKV; gather by byte equality; profile against a
 // token-by-token greedy written in the test, the closed form for identical heads, the end
 // points rho = 0 and 1, budget conservation and monotonicity in rho; lookup against a
-// hand-worked example.
+// hand-worked example; curves against the pinned selection (importance mass of M^pi(k)), a
+// library sort for the oracle metric, and closed forms.
 // No function here is "parity unpinned".
 //
 // Build: g++ -O2 -std=c++17 -ffp-contract=off -shared -fPIC lukv_oracle.cpp -o liblukv_oracle.so
@@ -394,6 +397,37 @@ int oracle_profile_budgets(const float* profile, const float* ratios, int R, int
 void oracle_select(const float* pooled, int n, int b, int32_t* kept) { select_head(pooled, n, b, 0, kept); }
 void oracle_select_sink(const float* pooled, int n, int b, int n_sink, int32_t* kept) {
   select_head(pooled, n, b, n_sink, kept);
+}
+
+// Utility-versus-budget curves of a proxy metric (Sec. 3.2: M^pi(k) is the set of the first k
+// positions when ranked by pi; Eq. "head_loss_def": the eviction loss of a retained set is the
+// oracle importance mass outside it).  U(k) = L(empty) - L(M^pi(k)) is the importance mass of
+// the k highest-ranked positions, i.e. the running sum of the importance in ranking order.
+// scores, importance: [heads][n] over the rankable positions; curves: [heads][P], point k =
+// U(min(k*s, n)), s = T/(P-1); running sum in fp64, each point rounded once to fp32.
+// Ranking as in the selection: sinks first, score descending, ties by lower position.
+void oracle_build_curves(const float* scores, const float* importance, int heads, int T, int w, int P, int n_sink,
+                         float* curves) {
+  const int n = T - w, s = T / (P - 1);
+  std::vector<int32_t> order(n);
+  std::vector<double> cum(n + 1);
+  for (int64_t u = 0; u < heads; ++u) {
+    // the ranking of select_head, kept in ranking order
+    std::iota(order.begin(), order.end(), 0);
+    const float* sc = scores + u * n;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t c) {
+      const bool sa = a < n_sink, sb = c < n_sink;
+      if (sa != sb) return sa;
+      if (sa) return false;
+      return sc[a] > sc[c];
+    });
+    cum[0] = 0.0;
+    for (int i = 0; i < n; ++i) cum[i + 1] = cum[i] + static_cast<double>(importance[u * n + order[i]]);
+    for (int k = 0; k < P; ++k) {
+      const int64_t b = std::min<int64_t>(static_cast<int64_t>(k) * s, n);
+      curves[u * P + k] = static_cast<float>(cum[b]);
+    }
+  }
 }
 
 // Selection + gather for all heads. scores: [S*N][n]; budgets: [S*N]; offsets: [S*N+1];

@@ -214,3 +214,14 @@ def profile_budgets(profile, ratios, T: int, w: int, sigma, min_keep: float = 0.
     if rc != 0:
         raise ValueError("sigma outside the ratio grid, or grid not strictly ascending")
     return budgets, offsets
+
+
+def build_curves(scores, importance, T: int, w: int, P: int, n_sink: int = 0) -> np.ndarray:
+    """Utility curves of the proxy ranking: scores, importance [heads][n] -> curves [heads][P] fp32."""
+    scores = _c(scores, np.float32)
+    importance = _c(importance, np.float32)
+    heads, n = scores.shape
+    assert n == T - w and importance.shape == scores.shape and T % (P - 1) == 0
+    curves = np.empty((heads, P), np.float32)
+    lib().oracle_build_curves(_p(scores), _p(importance), heads, T, w, P, int(n_sink), _p(curves))
+    return curves
