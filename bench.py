@@ -479,6 +479,15 @@ def run_profile_path(args):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / steps
 
+    # curves of the proxy ranking for all calibration queries at once (the queries are the batch)
+    pc = lukv.make_params(Mq, wl.L, wl.H, 1, 64, Tc, wl.w, 1, "fp32", Tc + 1)
+    g = torch.Generator(device="cuda").manual_seed(synth.BASE_SEED)
+    c_scores = torch.rand((Mq, wl.N, Tc - wl.w), generator=g, device="cuda")
+    c_imp = -torch.log1p(-torch.rand((Mq, wl.N, Tc - wl.w), generator=g, device="cuda"))
+    c_out = torch.empty((Mq, wl.N, Tc + 1), dtype=torch.float32, device="cuda")
+    curves_ms = timed(lambda: lukv.lukv_build_curves(pc, c_scores, c_imp, c_out), max(args.steps // 2, 1), 3)
+    del c_scores, c_imp, c_out
+
     build_ms = timed(lambda: lukv.lukv_profile_build(calib, U, Mq, ratios, phi, pws), args.steps, max(args.warmup, 3))
     build_launches = lukv.lukv_last_launch_count()
 
@@ -532,6 +541,8 @@ def run_profile_path(args):
                    "curve_points": Tc + 1, "ratios": R, "curve_bytes": int(U.numel() * 4)},
         "gpu_launches": build_launches * args.steps,
         "lookup": {"ms_per_call": lookup_ms, "sequences": wl.S, "heads": wl.N},
+        "build_curves": {"ms_per_call": curves_ms, "queries": Mq, "heads": wl.N, "positions": Tc - wl.w,
+                         "compares": float(Mq) * wl.N * (Tc - wl.w) ** 2},
         "online_mode": {"metric": METRIC, "value": wl.S * wl.T / (online_ms * 1e-3), "unit": UNIT,
                         "ms_per_step": online_ms, "packed_rows": rows, "launches_per_step": sum(counts),
                         "path_bytes_per_step": wl.S * wl.N * wl.T * wl.d * es + 2 * rows * wl.d * es},

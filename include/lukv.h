@@ -255,6 +255,28 @@ LUKV_API int lukv_profile_budgets(const lukv_params_t* params, const float* prof
                                   int32_t n_ratios, const float* sigma, int32_t* budgets, int32_t* offsets,
                                   void* stream);
 
+/*
+ * Utility-versus-budget curves of the proxy metric (Sec. 3.2: M^pi(k) is the set of the first k
+ * positions in the ranking of pi; Eq. "head_loss_def": the eviction loss of a retained set is the
+ * oracle importance mass outside it).  For every head, U(k) = L(empty) - L(M^pi(k)) is the
+ * importance mass of its k highest-ranked positions; the curve handed to stage (b) and to the
+ * profile build is U sampled every s = T/(P-1) tokens: curves[u][k] = U(min(k*s, n)).
+ * The ranking is the selection's (sinks first, score descending, lower position first among
+ * equals).  Sums are fp64 in ranking order, each point rounded once to fp32.  With S calibration
+ * queries as the batch, the output is the [n_queries][N][P] input of lukv_profile_build.
+ * The oracle importance itself (Eq. "oracle_importance") needs the model's decoding run and is an
+ * input here.
+ *
+ *   scores      [S][N][n] fp32   proxy scores of the rankable positions (lukv_score)
+ *   importance  [S][N][n] fp32   oracle importance of the same positions
+ *   curves      [S][N][P] fp32   out; curves[..][0] = 0, non-decreasing for importance >= 0
+ * Every position is ranked by counting the positions ahead of it (quadratic in n, no scratch
+ * memory), which suits calibration contexts of a few thousand tokens; n beyond about 24,000
+ * (8*n + 8*P bytes of shared memory above 200 KiB) returns LUKV_ERR_UNSUPPORTED.
+ */
+LUKV_API int lukv_build_curves(const lukv_params_t* params, const float* scores, const float* importance,
+                               float* curves, void* stream);
+
 /* Static description of a status code. */
 LUKV_API const char* lukv_strerror(int code);
 

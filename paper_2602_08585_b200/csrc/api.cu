@@ -468,6 +468,20 @@ int lukv_profile_budgets(const lukv_params_t* params, const float* profile, cons
   return LUKV_OK;
 }
 
+int lukv_build_curves(const lukv_params_t* params, const float* scores, const float* importance, float* curves,
+                      void* stream) {
+  Dims dm;
+  int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (!scores || !importance || !curves) return LUKV_ERR_INVALID_ARG;
+  if (curves_smem_bytes(dm.n, dm.P) > 200u * 1024u) return LUKV_ERR_UNSUPPORTED;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  if (launch_build_curves(dm, scores, importance, curves, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
+}
+
 const char* lukv_strerror(int code) {
   switch (code) {
     case LUKV_OK: return "ok";

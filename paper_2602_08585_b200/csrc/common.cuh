@@ -90,6 +90,10 @@ constexpr int kLookupSeqPerLaunch = 32;
 cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, const int* row_hi, const double* frac,
                                    int S, int N, int n, int w, int floor_tok, int32_t* budgets, int32_t* offsets,
                                    LaunchCtx& lc);
+// Curves of a proxy ranking: scores, importance [heads][n] -> curves [heads][P].
+size_t curves_smem_bytes(int n, int P);
+cudaError_t launch_build_curves(const Dims& dm, const float* scores, const float* importance, float* curves,
+                                LaunchCtx& lc);
 cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* budgets, const int32_t* offsets,
                           int32_t* kept_idx, int64_t rows_cap, HeadRange hr, LaunchCtx& lc);
 cudaError_t launch_gather(const Dims& dm, const int32_t* offsets, const int32_t* kept_idx, const void* k,

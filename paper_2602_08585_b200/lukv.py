@@ -22,7 +22,7 @@ DTYPE_BF16, DTYPE_FP32 = 0, 1
 
 EXPORTS = ("lukv_workspace_bytes", "lukv_score", "lukv_allocate", "lukv_select_gather", "lukv_compress",
            "lukv_strerror", "lukv_last_launch_count", "lukv_compress_profile", "lukv_allocate_static",
-           "lukv_profile_workspace_bytes", "lukv_profile_build", "lukv_profile_budgets")
+           "lukv_profile_workspace_bytes", "lukv_profile_build", "lukv_profile_budgets", "lukv_build_curves")
 
 
 class Params(ctypes.Structure):
@@ -77,6 +77,7 @@ def lib() -> ctypes.CDLL:
         L.lukv_profile_workspace_bytes.argtypes = [pp, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(sz)]
         L.lukv_profile_build.argtypes = [pp, vp, ctypes.c_int32, vp, ctypes.c_int32, vp, vp, sz, vp]
         L.lukv_profile_budgets.argtypes = [pp, vp, vp, ctypes.c_int32, vp, vp, vp, vp]
+        L.lukv_build_curves.argtypes = [pp, vp, vp, vp, vp]
         L.lukv_strerror.argtypes = [ctypes.c_int]
         L.lukv_strerror.restype = ctypes.c_char_p
         for name in EXPORTS[:5] + EXPORTS[6:]:
@@ -186,6 +187,12 @@ def lukv_profile_budgets(params: Params, profile, ratios, sigma, budgets, offset
     rc = lib().lukv_profile_budgets(ctypes.byref(params), _ptr(profile), r.ctypes.data, int(r.shape[0]),
                                     sg.ctypes.data, _ptr(budgets), _ptr(offsets), _stream(stream))
     return _check(rc, "lukv_profile_budgets", check)
+
+
+def lukv_build_curves(params: Params, scores, importance, curves, stream=None, check: bool = True) -> int:
+    """Curves of the proxy ranking: scores, importance [S][N][n] -> curves [S][N][P] (all device)."""
+    rc = lib().lukv_build_curves(ctypes.byref(params), _ptr(scores), _ptr(importance), _ptr(curves), _stream(stream))
+    return _check(rc, "lukv_build_curves", check)
 
 
 def lukv_select_gather(params: Params, scores, budgets, offsets, k, v, k_out, v_out, kept_idx, rows_cap: int, ws,
