@@ -48,7 +48,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0,
                     help="override the workload's layer count (a reduced case for profiler captures)")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-heads", type=int, default=24, help="heads in the CPU-baseline sample")
+    ap.add_argument("--cpu-heads", type=int, default=48, help="heads in the CPU-baseline sample")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
