@@ -22,6 +22,8 @@
 //   gather   : the retained index set I of Sec. 3.2 materialised as a packed cache.
 //   curves   : utility-versus-budget curve of a proxy metric = running sum of the oracle
 //              importance in the metric's ranking order (Sec. 3.2, Eq. "head_loss_def").
+//   exact    : the allocation problem on the raw curves by the multiple-choice-knapsack
+//              recursion (Sec. 4.2 mentions the exact solver as the comparison point).
 //   deployment settings (App. E): attention sinks always ranked first; a minimum number of
 //              tokens per head handed out before the greedy starts.  Both default to off.
 //   profile  : offline profile = mean over calibration queries of the optimal local ratios
@@ -36,7 +38,8 @@
 // token-by-token greedy written in the test, the closed form for identical heads, the end
 // points rho = 0 and 1, budget conservation and monotonicity in rho; lookup against a
 // hand-worked example; curves against the pinned selection (importance mass of M^pi(k)), a
-// library sort for the oracle metric, and closed forms.
+// library sort for the oracle metric, and closed forms; the exact solver against exhaustive
+// search, against the greedy on concave curves, and between the greedy's raw and hull values.
 // No function here is "parity unpinned".
 //
 // Build: g++ -O2 -std=c++17 -ffp-contract=off -shared -fPIC lukv_oracle.cpp -o liblukv_oracle.so
@@ -46,6 +49,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <limits>
 #include <numeric>
 #include <vector>
 
@@ -397,6 +401,53 @@ int oracle_profile_budgets(const float* profile, const float* ratios, int R, int
 void oracle_select(const float* pooled, int n, int b, int32_t* kept) { select_head(pooled, n, b, 0, kept); }
 void oracle_select_sink(const float* pooled, int n, int b, int n_sink, int32_t* kept) {
   select_head(pooled, n, b, n_sink, kept);
+}
+
+// Exact solution of the allocation problem (Sec. 4.2, Eq. "combinatorial_optimization": maximise
+// the summed utility -- minimise the summed loss -- over integer budgets with sum b = B), on the
+// curves as given (no relaxation), by dynamic programming over the heads: the classic
+// multiple-choice-knapsack recursion f_h(x) = max_b f_{h-1}(x-b) + U_h(b).  Token-resolution
+// curves only (P = T+1, point b = utility of keeping b tokens, 0 <= b <= n).  fp64.
+// budgets: [S][N] one optimal solution (the smallest b on ties, heads taken last to first);
+// values: [S] the optimum.  Returns 0, or -1 for s != 1 or a budget outside [0, N*n].
+int oracle_exact_allocate(const float* curves, int N, int P, int T, int w, int S, const int64_t* budgets_in,
+                          int32_t* budgets, double* values) {
+  const int64_t n = T - w;
+  if (P != T + 1) return -1;
+  const double ninf = -std::numeric_limits<double>::infinity();
+  for (int q = 0; q < S; ++q) {
+    const int64_t B = budgets_in[q];
+    if (B < 0 || B > static_cast<int64_t>(N) * n) return -1;
+    std::vector<double> f(B + 1, ninf), g(B + 1);
+    std::vector<int32_t> choice(static_cast<size_t>(N) * (B + 1));
+    f[0] = 0.0;
+    for (int h = 0; h < N; ++h) {
+      const float* U = curves + static_cast<size_t>(h) * P;
+      for (int64_t x = 0; x <= B; ++x) {
+        double best = ninf;
+        int32_t arg = 0;
+        const int64_t bmax = std::min<int64_t>(x, n);
+        for (int64_t b = 0; b <= bmax; ++b) {
+          const double v = f[x - b] + static_cast<double>(U[b]);
+          if (v > best) {
+            best = v;
+            arg = static_cast<int32_t>(b);
+          }
+        }
+        g[x] = best;
+        choice[static_cast<size_t>(h) * (B + 1) + x] = arg;
+      }
+      f.swap(g);
+    }
+    values[q] = f[B];
+    int64_t x = B;
+    for (int h = N - 1; h >= 0; --h) {
+      const int32_t b = choice[static_cast<size_t>(h) * (B + 1) + x];
+      budgets[static_cast<size_t>(q) * N + h] = b;
+      x -= b;
+    }
+  }
+  return 0;
 }
 
 // Utility-versus-budget curves of a proxy metric (Sec. 3.2: M^pi(k) is the set of the first k

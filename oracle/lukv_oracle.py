@@ -43,6 +43,7 @@ def lib() -> ctypes.CDLL:
         for name in ("oracle_allocate_floor", "oracle_compress_ext", "oracle_profile_build_floor",
                      "oracle_profile_budgets_floor"):
             getattr(_lib, name).restype = ctypes.c_int
+        _lib.oracle_exact_allocate.restype = ctypes.c_int
         _lib.oracle_floor_tokens.restype = ctypes.c_int64
         _lib.oracle_floor_tokens.argtypes = [ctypes.c_float, ctypes.c_int]
     return _lib
@@ -225,3 +226,17 @@ def build_curves(scores, importance, T: int, w: int, P: int, n_sink: int = 0) ->
     curves = np.empty((heads, P), np.float32)
     lib().oracle_build_curves(_p(scores), _p(importance), heads, T, w, P, int(n_sink), _p(curves))
     return curves
+
+
+def exact_allocate(curves, T: int, w: int, budgets_in):
+    """Exact allocation on token-resolution curves [N][T+1] -> (budgets [S][N] int32, optimum values [S] float64)."""
+    curves = _c(curves, np.float32)
+    budgets_in = _c(budgets_in, np.int64)
+    N, P = curves.shape
+    S = budgets_in.shape[0]
+    budgets = np.empty((S, N), np.int32)
+    values = np.empty(S, np.float64)
+    rc = lib().oracle_exact_allocate(_p(curves), N, P, T, w, S, _p(budgets_in), _p(budgets), _p(values))
+    if rc != 0:
+        raise ValueError("needs token-resolution curves (P = T+1) and budgets in [0, N*(T-w)]")
+    return budgets, values
