@@ -491,6 +491,21 @@ def run_profile_path(args):
     build_ms = timed(lambda: lukv.lukv_profile_build(calib, U, Mq, ratios, phi, pws), args.steps, max(args.warmup, 3))
     build_launches = lukv.lukv_last_launch_count()
 
+    # exact solver on the first query's curves at 70 % compression, beside the greedy on the same curves
+    Bx = int(0.3 * wl.N * (Tc - wl.w))
+    xws = torch.empty(lukv.lukv_exact_workspace_bytes(calib, Bx), dtype=torch.uint8, device="cuda")
+    xb = torch.empty((1, wl.N), dtype=torch.int32, device="cuda")
+    xo = torch.empty((wl.N + 1,), dtype=torch.int32, device="cuda")
+    xv = torch.zeros(1, dtype=torch.float64, device="cuda")
+    exact_ms = timed(lambda: lukv.lukv_exact_allocate(calib, U[0], [Bx], xb, xo, xv, xws), 3, 1)
+    exact_launches = lukv.lukv_last_launch_count()
+    gb = torch.empty((1, wl.N), dtype=torch.int32, device="cuda")
+    aws = lukv.alloc_workspace(calib)
+    lukv.lukv_allocate(calib, U[0], [Bx], gb, xo, aws)
+    greedy_raw = float(U[0].double().gather(1, gb[0].long()[:, None]).sum().item())
+    exact_val = float(xv.item())
+    del xws, aws
+
     p = lukv.make_params(wl.S, wl.L, wl.H, wl.G, wl.d, wl.T, wl.w, wl.kp, wl.dtype, wl.P)
     q, k, v = synth.gen_tensors(wl, "cuda")
     ws = lukv.alloc_workspace(p)
@@ -541,6 +556,9 @@ def run_profile_path(args):
                    "curve_points": Tc + 1, "ratios": R, "curve_bytes": int(U.numel() * 4)},
         "gpu_launches": build_launches * args.steps,
         "lookup": {"ms_per_call": lookup_ms, "sequences": wl.S, "heads": wl.N},
+        "exact_allocate": {"ms_per_call": exact_ms, "heads": wl.N, "positions": Tc - wl.w, "budget": Bx,
+                           "launches": exact_launches, "optimum": exact_val, "greedy_on_raw_curves": greedy_raw,
+                           "relaxation_gap": (exact_val - greedy_raw) / exact_val},
         "build_curves": {"ms_per_call": curves_ms, "queries": Mq, "heads": wl.N, "positions": Tc - wl.w,
                          "compares": float(Mq) * wl.N * (Tc - wl.w) ** 2},
         "online_mode": {"metric": METRIC, "value": wl.S * wl.T / (online_ms * 1e-3), "unit": UNIT,

@@ -277,6 +277,28 @@ LUKV_API int lukv_profile_budgets(const lukv_params_t* params, const float* prof
 LUKV_API int lukv_build_curves(const lukv_params_t* params, const float* scores, const float* importance,
                                float* curves, void* stream);
 
+/*
+ * Exact allocation (Sec. 4.2, Eq. "combinatorial_optimization": maximise the summed utility over
+ * integer budgets with sum b = B on the curves as given, no relaxation; the paper names the exact
+ * solver as the comparison point of its relaxation).  A tool for cross-checks, not part of the
+ * hot path: the multiple-choice-knapsack recursion over the heads, N*B*n/2 additions in fp32, one
+ * launch per head.  Token-resolution curves only (P = T+1, so s = 1), n <= 65535, min_keep = 0;
+ * anything else is LUKV_ERR_UNSUPPORTED.
+ *
+ *   curves      [N][P] fp32          as in lukv_allocate (need not be monotone or concave)
+ *   budgets_in  [S] int64, HOST      0 <= B_q <= N*n
+ *   budgets     [S][N] int32         out: one optimal solution (ties: the smallest budget for the
+ *                                    later head); sum_hid budgets[q][hid] == B_q
+ *   offsets     [S*N+1] int32        out, as in lukv_allocate
+ *   values      [S] fp64             out: the optimum (accumulated in fp32)
+ *   ws          lukv_exact_workspace_bytes(params, max_q B_q) bytes, 256-byte aligned:
+ *               two fp32 rows of B+1 values and the 16-bit argmax of every (head, budget)
+ */
+LUKV_API int lukv_exact_workspace_bytes(const lukv_params_t* params, int64_t max_budget, size_t* bytes /* HOST, out */);
+LUKV_API int lukv_exact_allocate(const lukv_params_t* params, const float* curves, const int64_t* budgets_in,
+                                 int32_t* budgets, int32_t* offsets, double* values, void* ws, size_t ws_bytes,
+                                 void* stream);
+
 /* Static description of a status code. */
 LUKV_API const char* lukv_strerror(int code);
 

@@ -482,6 +482,43 @@ int lukv_build_curves(const lukv_params_t* params, const float* scores, const fl
   return LUKV_OK;
 }
 
+// Token resolution, no minimum retention: what the exact solver covers.
+static int make_exact_dims(const lukv_params_t* params, Dims* dm) {
+  const int rc = make_dims(params, dm);
+  if (rc != LUKV_OK) return rc;
+  if (dm->seg != 1 || dm->floor_tok != 0 || dm->n > 65535) return LUKV_ERR_UNSUPPORTED;
+  return LUKV_OK;
+}
+
+int lukv_exact_workspace_bytes(const lukv_params_t* params, int64_t max_budget, size_t* bytes) {
+  Dims dm;
+  if (!bytes) return LUKV_ERR_INVALID_ARG;
+  const int rc = make_exact_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (max_budget < 0 || max_budget > (int64_t)dm.N * dm.n) return LUKV_ERR_BUDGET;
+  *bytes = exact_workspace_bytes(dm, max_budget);
+  return LUKV_OK;
+}
+
+int lukv_exact_allocate(const lukv_params_t* params, const float* curves, const int64_t* budgets_in, int32_t* budgets,
+                        int32_t* offsets, double* values, void* ws, size_t ws_bytes, void* stream) {
+  Dims dm;
+  int rc = make_exact_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (!curves || !budgets_in || !budgets || !offsets || !values || !ws || (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return LUKV_ERR_INVALID_ARG;
+  int64_t rows, bmax = 0;
+  if ((rc = check_budgets(dm, budgets_in, &rows)) != LUKV_OK) return rc;
+  if (rows >= (int64_t)1 << 31) return LUKV_ERR_UNSUPPORTED;
+  for (int q = 0; q < dm.S; ++q) bmax = budgets_in[q] > bmax ? budgets_in[q] : bmax;
+  if (ws_bytes < exact_workspace_bytes(dm, bmax)) return LUKV_ERR_WORKSPACE_TOO_SMALL;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  if (launch_exact_allocate(dm, curves, budgets_in, budgets, offsets, values, ws, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
+}
+
 const char* lukv_strerror(int code) {
   switch (code) {
     case LUKV_OK: return "ok";

@@ -94,6 +94,10 @@ cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, cons
 size_t curves_smem_bytes(int n, int P);
 cudaError_t launch_build_curves(const Dims& dm, const float* scores, const float* importance, float* curves,
                                 LaunchCtx& lc);
+// Exact allocation (dynamic programme over the heads) at token resolution.
+size_t exact_workspace_bytes(const Dims& dm, int64_t max_budget);
+cudaError_t launch_exact_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, int32_t* budgets,
+                                  int32_t* offsets, double* values, void* ws, LaunchCtx& lc);
 cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* budgets, const int32_t* offsets,
                           int32_t* kept_idx, int64_t rows_cap, HeadRange hr, LaunchCtx& lc);
 cudaError_t launch_gather(const Dims& dm, const int32_t* offsets, const int32_t* kept_idx, const void* k,

@@ -22,7 +22,8 @@ DTYPE_BF16, DTYPE_FP32 = 0, 1
 
 EXPORTS = ("lukv_workspace_bytes", "lukv_score", "lukv_allocate", "lukv_select_gather", "lukv_compress",
            "lukv_strerror", "lukv_last_launch_count", "lukv_compress_profile", "lukv_allocate_static",
-           "lukv_profile_workspace_bytes", "lukv_profile_build", "lukv_profile_budgets", "lukv_build_curves")
+           "lukv_profile_workspace_bytes", "lukv_profile_build", "lukv_profile_budgets", "lukv_build_curves", "lukv_exact_workspace_bytes",
+           "lukv_exact_allocate")
 
 
 class Params(ctypes.Structure):
@@ -78,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.lukv_profile_build.argtypes = [pp, vp, ctypes.c_int32, vp, ctypes.c_int32, vp, vp, sz, vp]
         L.lukv_profile_budgets.argtypes = [pp, vp, vp, ctypes.c_int32, vp, vp, vp, vp]
         L.lukv_build_curves.argtypes = [pp, vp, vp, vp, vp]
+        L.lukv_exact_workspace_bytes.argtypes = [pp, i64, ctypes.POINTER(sz)]
+        L.lukv_exact_allocate.argtypes = [pp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.lukv_strerror.argtypes = [ctypes.c_int]
         L.lukv_strerror.restype = ctypes.c_char_p
         for name in EXPORTS[:5] + EXPORTS[6:]:
@@ -193,6 +196,24 @@ def lukv_build_curves(params: Params, scores, importance, curves, stream=None, c
     """Curves of the proxy ranking: scores, importance [S][N][n] -> curves [S][N][P] (all device)."""
     rc = lib().lukv_build_curves(ctypes.byref(params), _ptr(scores), _ptr(importance), _ptr(curves), _stream(stream))
     return _check(rc, "lukv_build_curves", check)
+
+
+def lukv_exact_workspace_bytes(params: Params, max_budget: int) -> int:
+    out = ctypes.c_size_t(0)
+    rc = lib().lukv_exact_workspace_bytes(ctypes.byref(params), int(max_budget), ctypes.byref(out))
+    if rc != OK:
+        raise LukvError(rc, "lukv_exact_workspace_bytes")
+    return int(out.value)
+
+
+def lukv_exact_allocate(params: Params, curves, budgets_in, budgets, offsets, values, ws, stream=None,
+                        check: bool = True) -> int:
+    """Exact allocation on token-resolution curves; values is a float64 device tensor [S]."""
+    b = _host_budgets(budgets_in)
+    rc = lib().lukv_exact_allocate(ctypes.byref(params), _ptr(curves), b.ctypes.data, _ptr(budgets), _ptr(offsets),
+                                   _ptr(values), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                   _stream(stream))
+    return _check(rc, "lukv_exact_allocate", check)
 
 
 def lukv_select_gather(params: Params, scores, budgets, offsets, k, v, k_out, v_out, kept_idx, rows_cap: int, ws,
