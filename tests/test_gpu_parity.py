@@ -237,3 +237,26 @@ def test_compress_is_deterministic():
     b = gpu_compress(params_of(wl), q, k, v, curves, wl.budgets())
     assert torch.equal(a.kept_idx, b.kept_idx) and torch.equal(a.k_out.view(torch.int16), b.k_out.view(torch.int16))
     assert torch.equal(a.budgets, b.budgets) and torch.equal(a.offsets, b.offsets)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(L=2, H=4, T=8192, P=129),                         # 128 query rows per head: one row block
+    dict(L=1, H=3, G=7, T=6000 + 96, w=32, P=2),           # 224 query rows: two row blocks, ragged last key tile
+    dict(S=3, L=1, H=5, T=3000 + 40, w=40, kp=5, P=2),     # 160 rows, several sequences, short items
+    dict(L=1, H=40, T=1024, P=2),                          # fewer work items than CTAs per head
+])
+def test_tensor_core_scorer_repeats_bit_for_bit(kw):
+    """The persistent scorer's CTAs hand partial results to one another; a rare ordering bug there shows as a
+    repetition whose bits differ.  Every reduction has a fixed order, so 40 repetitions must be identical."""
+    wl = synth.scaled(synth.CONFIGS["llama8b_1layer_8k"], needles=16, **kw)
+    p = params_of(wl)
+    q, k, _ = synth.gen_tensors(wl, "cuda")
+    ws = lukv.alloc_workspace(p)
+    first = torch.empty((p.batch, p.N, p.n), dtype=torch.float32, device="cuda")
+    lukv.lukv_score(p, q, k, first, ws)
+    again = torch.empty_like(first)
+    for rep in range(40):
+        again.fill_(-1.0)
+        lukv.lukv_score(p, q, k, again, ws)
+        assert torch.equal(again, first), rep
+    assert torch.isfinite(first).all() and (first >= 0).all()
