@@ -230,6 +230,36 @@ __device__ __forceinline__ uint64_t ex2_pair(uint64_t x) {
   unpack2(x, a, b);
   return pack2(ex2(a), ex2(b));
 }
+#ifndef LUKV_POLY_SEL1
+#define LUKV_POLY_SEL1(i) ((((i) >> 2) & 3) == 0)
+#endif
+#ifndef LUKV_POLY_SEL2
+#define LUKV_POLY_SEL2(i) ((((i) >> 2) & 3) == 0)
+#endif
+// both lanes of a packed pair through the FMA-pipe polynomial (integer part into the exponent field)
+__device__ __forceinline__ uint64_t ex2_poly_pair(uint64_t x) {
+  float a, b;
+  unpack2(x, a, b);
+  // the exponent field has room for [-126, 126]; arguments outside saturate there, which keeps the two
+  // properties the callers rely on: masked (-inf) terms stay negligible (2^-126), and terms too large for the
+  // running reference (including +inf) still push the chunk sum past the re-referencing threshold
+  x = pack2(fminf(fmaxf(a, -126.f), 126.f), fminf(fmaxf(b, -126.f), 126.f));
+  const uint64_t magic = pack2(12582912.f, 12582912.f), nmagic = pack2(-12582912.f, -12582912.f);
+  const uint64_t t = fadd2(x, magic);
+  float ta, tb, sa, sb;
+  unpack2(t, ta, tb);
+  unpack2(fadd2(t, nmagic), sa, sb);
+  const uint64_t f = fadd2(x, pack2(-sa, -sb));
+  uint64_t p = pack2(0.009570101276040077f, 0.009570101276040077f);
+  p = ffma2(p, f, pack2(0.05591785907745361f, 0.05591785907745361f));
+  p = ffma2(p, f, pack2(0.240247443318367f, 0.240247443318367f));
+  p = ffma2(p, f, pack2(0.6931217908859253f, 0.6931217908859253f));
+  p = ffma2(p, f, pack2(0.9999992847442627f, 0.9999992847442627f));
+  float pa, pb;
+  unpack2(p, pa, pb);
+  return pack2(__int_as_float(__float_as_int(pa) + (__float_as_int(ta) << 23)),
+               __int_as_float(__float_as_int(pb) + (__float_as_int(tb) << 23)));
+}
 __device__ __forceinline__ float sum4(uint64_t p, uint64_t q) {
   float a, b, c, d;
   unpack2(p, a, b);
@@ -348,7 +378,8 @@ __device__ __forceinline__ void p1_chunk(const float (&v)[32], int jbase, int li
 #pragma unroll
   for (int i = 0; i < 32; i += 4) {
     acc0 = fadd2(acc0, ex2_pair(ffma2(pack2(x[i], x[i + 1]), sc2, nm2)));
-    acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(x[i + 2], x[i + 3]), sc2, nm2)));
+    if (LUKV_POLY_SEL1(i)) acc1 = fadd2(acc1, ex2_poly_pair(ffma2(pack2(x[i + 2], x[i + 3]), sc2, nm2)));
+    else acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(x[i + 2], x[i + 3]), sc2, nm2)));
   }
   const float cs = sum4(acc0, acc1);
   if (cs <= 1e12f) {  // false for inf and NaN
@@ -377,7 +408,8 @@ __device__ __forceinline__ void p2_chunk(const float (&v)[32], const float* nlse
   for (int i = 0; i < 32; i += 4) {
     const ulonglong2 ls = *reinterpret_cast<const ulonglong2*>(nlse + i);  // (-lse[i], -lse[i+1]), (-lse[i+2], -lse[i+3])
     acc0 = fadd2(acc0, ex2_pair(ffma2(pack2(v[i], v[i + 1]), sc2, ls.x)));
-    acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(v[i + 2], v[i + 3]), sc2, ls.y)));
+    if (LUKV_POLY_SEL2(i)) acc1 = fadd2(acc1, ex2_poly_pair(ffma2(pack2(v[i + 2], v[i + 3]), sc2, ls.y)));
+    else acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(v[i + 2], v[i + 3]), sc2, ls.y)));
   }
 }
 
