@@ -237,13 +237,16 @@ __device__ __forceinline__ uint64_t ex2_pair(uint64_t x) {
 #define LUKV_POLY_SEL2(i) ((((i) >> 2) & 3) == 0)
 #endif
 // both lanes of a packed pair through the FMA-pipe polynomial (integer part into the exponent field)
+template <bool UPPER>
 __device__ __forceinline__ uint64_t ex2_poly_pair(uint64_t x) {
   float a, b;
   unpack2(x, a, b);
   // the exponent field has room for [-126, 126]; arguments outside saturate there, which keeps the two
   // properties the callers rely on: masked (-inf) terms stay negligible (2^-126), and terms too large for the
   // running reference (including +inf) still push the chunk sum past the re-referencing threshold
-  x = pack2(fminf(fmaxf(a, -126.f), 126.f), fminf(fmaxf(b, -126.f), 126.f));
+  // (UPPER = false: the caller keeps the arguments below the upper end itself)
+  x = UPPER ? pack2(fminf(fmaxf(a, -126.f), 126.f), fminf(fmaxf(b, -126.f), 126.f))
+            : pack2(fmaxf(a, -126.f), fmaxf(b, -126.f));
   const uint64_t magic = pack2(12582912.f, 12582912.f), nmagic = pack2(-12582912.f, -12582912.f);
   const uint64_t t = fadd2(x, magic);
   float ta, tb, sa, sb;
@@ -375,14 +378,21 @@ __device__ __forceinline__ void p1_chunk(const float (&v)[32], int jbase, int li
   for (int i = 0; i < 32; ++i) x[i] = (!MASKED || jbase + i <= lim) ? v[i] : -INFINITY;
   const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m, -m);
   uint64_t acc0 = 0ull, acc1 = 0ull;  // bit pattern of (+0, +0)
+  // The polynomial has no overflow of its own (its exponent arithmetic wraps), so the largest argument that
+  // goes through it is checked once per chunk instead: it joins the test that sends the chunk to the exact path.
+  float pmax = -INFINITY;
 #pragma unroll
   for (int i = 0; i < 32; i += 4) {
     acc0 = fadd2(acc0, ex2_pair(ffma2(pack2(x[i], x[i + 1]), sc2, nm2)));
-    if (LUKV_POLY_SEL1(i)) acc1 = fadd2(acc1, ex2_poly_pair(ffma2(pack2(x[i + 2], x[i + 3]), sc2, nm2)));
-    else acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(x[i + 2], x[i + 3]), sc2, nm2)));
+    if (LUKV_POLY_SEL1(i)) {
+      pmax = fmaxf(pmax, fmaxf(x[i + 2], x[i + 3]));
+      acc1 = fadd2(acc1, ex2_poly_pair<false>(ffma2(pack2(x[i + 2], x[i + 3]), sc2, nm2)));
+    } else {
+      acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(x[i + 2], x[i + 3]), sc2, nm2)));
+    }
   }
   const float cs = sum4(acc0, acc1);
-  if (cs <= 1e12f) {  // false for inf and NaN
+  if (cs <= 1e12f && fmaf(pmax, scale_log2, -m) <= 100.f) {  // false for inf and NaN
     l += cs;
     return;
   }
@@ -408,7 +418,7 @@ __device__ __forceinline__ void p2_chunk(const float (&v)[32], const float* nlse
   for (int i = 0; i < 32; i += 4) {
     const ulonglong2 ls = *reinterpret_cast<const ulonglong2*>(nlse + i);  // (-lse[i], -lse[i+1]), (-lse[i+2], -lse[i+3])
     acc0 = fadd2(acc0, ex2_pair(ffma2(pack2(v[i], v[i + 1]), sc2, ls.x)));
-    if (LUKV_POLY_SEL2(i)) acc1 = fadd2(acc1, ex2_poly_pair(ffma2(pack2(v[i + 2], v[i + 3]), sc2, ls.y)));
+    if (LUKV_POLY_SEL2(i)) acc1 = fadd2(acc1, ex2_poly_pair<false>(ffma2(pack2(v[i + 2], v[i + 3]), sc2, ls.y)));
     else acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(v[i + 2], v[i + 3]), sc2, ls.y)));
   }
 }
