@@ -136,7 +136,7 @@ static SideStream* side_stream() {
 
 // The whole path.  Allocation depends only on the curves, scoring only on Q/K; selection needs
 // both, the gather follows.  With `overlap` the two allocation kernels run on an auxiliary stream
-// beside the scorer, which then leaves two SMs to them (its CTAs fill theirs completely); the
+// beside the scorer, which then leaves one SM to them (its CTAs fill theirs completely); the
 // caller's stream waits for the budgets before selection, so stream order is preserved.
 static int run_compress(const Dims& dm, const void* q_win, const void* k, const void* v, const float* curves,
                         const int64_t* budgets_in, void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets,
@@ -154,7 +154,7 @@ static int run_compress(const Dims& dm, const void* q_win, const void* k, const 
     if (launch_allocate(dm, curves, budgets_in, w.gains, budgets, offsets, ls) != cudaSuccess) rc = LUKV_ERR_CUDA;
     if (cudaEventRecord(side->join, ls.st) != cudaSuccess) rc = LUKV_ERR_CUDA;
     lc.launches += ls.launches;
-    if (rc == LUKV_OK && (launch_score_tc(dm, q_win, k, w, dev_status, all_heads(dm), true, 2, lc) != cudaSuccess ||
+    if (rc == LUKV_OK && (launch_score_tc(dm, q_win, k, w, dev_status, all_heads(dm), true, 1, lc) != cudaSuccess ||
                           launch_pool(dm, w.raw, w.pooled, all_heads(dm), lc) != cudaSuccess))
       rc = LUKV_ERR_CUDA;
     // join even after a failure: the caller's stream must not run ahead of work already enqueued

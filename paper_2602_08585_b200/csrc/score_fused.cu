@@ -328,6 +328,7 @@ struct FusedArgs {
   int lse_rows;        // M rounded up to a multiple of 4
   int head0, nheads;   // heads [head0, head0+nheads) are scored by this launch
   int item_tiles, items_per_head, tiles_T, tiles_n;
+  int adapt_items;     // host only: let the launcher pick a multiple of item_tiles
   int npad;            // pass 2: query rows rounded up to a multiple of 32 (MMA N and columns read)
   int lag;             // 2..kMaxLag: pass 1 of item k+lag-1 precedes pass 2 of item k
   int l2_hints;        // 1: pass-1 key loads ask L2 to keep the lines, pass-2 loads to drop them first
@@ -916,6 +917,27 @@ cudaError_t launch_fused(const CUtensorMap& qm, const CUtensorMap& km, FusedArgs
   if (spare_sms > 0 && sms > 8 * spare_sms) sms -= spare_sms;
   // A CTA runs pass 1 of later items before pass 2 of the current one, so a head's items must
   // not outnumber the CTAs (else a CTA would wait for partials that it is due to produce itself).
+  if (args.adapt_items) {
+    // Larger work items mean fewer job changes and fewer partials to fold per head, but coarser dealing.
+    // A CTA's critical path is its number of items times (tiles per item + about one tile's time of
+    // per-item overhead); measured on 256 heads x 256 tiles and 148 CTAs: 0.89 ms with 8 tiles per item,
+    // 0.84 with 16, 0.82 with 32.  The price of large items is that pass 2 no longer finds all its key
+    // tiles in L2; the kernel is bound by the exp2 unit, not by HBM, so re-reading part of K costs nothing.
+    int best = args.item_tiles;
+    double best_cost = 1e30;
+    for (int mult = 1; mult <= 4; mult *= 2) {
+      const int it = args.item_tiles * mult;
+      const long long per_head = (args.tiles_T + it - 1) / it;
+      const long long items = (long long)args.nheads * per_head;
+      const long long ctas = items < sms ? items : sms;
+      const double cost = (double)((items + ctas - 1) / ctas) * (it + 1.05);
+      if (cost < best_cost * 0.995) {
+        best_cost = cost;
+        best = it;
+      }
+    }
+    args.item_tiles = best;
+  }
   while ((args.tiles_T + args.item_tiles - 1) / args.item_tiles > sms) ++args.item_tiles;
   args.items_per_head = (args.tiles_T + args.item_tiles - 1) / args.item_tiles;
   const int total_items = args.nheads * args.items_per_head;
@@ -978,8 +1000,9 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
   args.lse_rows = (dm.M + 3) & ~3;
   args.head0 = hr.h0;
   args.nheads = hr.nh;
-  args.item_tiles = score_item_tiles();
   args.tiles_T = (dm.T + kTileKeys - 1) / kTileKeys;
+  args.item_tiles = score_item_tiles();
+  args.adapt_items = getenv("LUKV_ITEM_TILES") ? 0 : 1;
   args.tiles_n = (dm.n + kTileKeys - 1) / kTileKeys;
   args.items_per_head = 0;  // set by the launcher
   args.npad = (dm.M + 31) & ~31;
