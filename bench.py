@@ -314,7 +314,8 @@ def run_ours(args):
         peak_exp = 16.0 * sms * (sampler.max_mhz or 1965) * 1e6 / 1e9
         roofline = {"kernel": dom, "bound": "alu", "achieved": exps / dom_s / 1e9, "peak": peak_exp,
                     "unit": "Gexp2/s", "frac": exps / dom_s / 1e9 / peak_exp,
-                    "peak_source": "16 exp2 per clock per SM x SM count x max SM clock",
+                    "peak_source": "16 exp2 per clock per SM (special-function unit) x SM count x max SM clock; one exp2 pair in "
+                                   "eight is evaluated on the FMA pipe instead, so the ceiling is 8/7 of it",
                     "algorithmic_exp2_per_launch": exps, "algorithmic_bytes_per_launch": dom_bytes,
                     "hbm_achieved_gbs": dom_gbs, "hbm_peak_gbs": peak, "hbm_frac": dom_gbs / peak,
                     "hbm_peak_source": peak_src, "traffic": load_traffic(dom, wl.name)}
