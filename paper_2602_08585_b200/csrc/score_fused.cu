@@ -921,11 +921,11 @@ cudaError_t launch_fused(const CUtensorMap& qm, const CUtensorMap& km, FusedArgs
     // Larger work items mean fewer job changes and fewer partials to fold per head, but coarser dealing.
     // A CTA's critical path is its number of items times (tiles per item + about one tile's time of
     // per-item overhead); measured on 256 heads x 256 tiles and 148 CTAs: 0.89 ms with 8 tiles per item,
-    // 0.84 with 16, 0.82 with 32.  The price of large items is that pass 2 no longer finds all its key
+    // 0.84 with 16, 0.82 with 32, 0.81 with 64.  The price of large items is that pass 2 no longer finds all its key
     // tiles in L2; the kernel is bound by the exp2 unit, not by HBM, so re-reading part of K costs nothing.
     int best = args.item_tiles;
     double best_cost = 1e30;
-    for (int mult = 1; mult <= 4; mult *= 2) {
+    for (int mult = 1; mult <= 8; mult *= 2) {
       const int it = args.item_tiles * mult;
       const long long per_head = (args.tiles_T + it - 1) / it;
       const long long items = (long long)args.nheads * per_head;
