@@ -7,6 +7,11 @@
  *   select    per-head top-b positions by score
  *   gather    compact the kept K/V rows (plus the always-kept observation window)
  *
+ * Beside the four stages the library has the paper's profile mode (lukv_profile_build,
+ * lukv_profile_budgets: Sec. 4.3), the curve builder that feeds it (lukv_build_curves), an
+ * exact solver for cross-checks (lukv_exact_allocate) and a variant of the allocation that needs
+ * no caller scratch (lukv_allocate_static).
+ *
  * Problem statement implemented (paper Sec. 4.2 Eq. "combinatorial_optimization" and its
  * relaxed form, Sec. 4.3 "Online Execution"): given per-head utility-versus-budget
  * curves, a global budget and the prefill KV cache, produce integer per-head budgets b
