@@ -176,7 +176,12 @@ __global__ void __launch_bounds__(kGreedyMaxThreads) greedy_kernel(const float* 
   }
   // (each thread only ever touches the heads it owns, so lo/hi/mid need no barrier of their own)
   if (!all_taken) {
+    // the low key word is k*N + hid < N*(P-1): its bits from idx_bits up are zero in every key, a pass over
+    // them would change nothing
+    int idx_bits = 0;
+    while (idx_bits < 32 && ((unsigned long long)N * (unsigned)G1) >> idx_bits) ++idx_bits;
     for (int bit = 63; bit >= 0; --bit) {
+      if (bit < 32 && bit >= idx_bits) continue;
       long long local = 0;
       for (int h = tid; h < N; h += nthr) {
         const int l = lo[h], r = hi[h];
