@@ -260,3 +260,15 @@ def test_tensor_core_scorer_repeats_bit_for_bit(kw):
         lukv.lukv_score(p, q, k, again, ws)
         assert torch.equal(again, first), rep
     assert torch.isfinite(first).all() and (first >= 0).all()
+
+
+def test_allocate_more_heads_than_threads(oracle):
+    # 1500 heads: the allocation CTA (at most 1024 threads, one head each) loops over the heads
+    rng = np.random.default_rng(9)
+    N, P, T, w = 1500, 17, 256, 16
+    inc = rng.exponential(size=(N, P - 1)) * np.where(rng.random((N, P - 1)) < 0.2, 3.0, 1.0)
+    U = np.zeros((N, P), np.float32)
+    U[:, 1:] = np.cumsum(inc, axis=1)
+    U[::7] = U[3]                        # many identical heads: ties across heads
+    n = T - w
+    _alloc_case(oracle, N, P, T, w, U, [0, 1, 12345, N * n // 3, N * n - 1, N * n], L=3)
