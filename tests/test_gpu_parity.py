@@ -272,3 +272,32 @@ def test_allocate_more_heads_than_threads(oracle):
     U[::7] = U[3]                        # many identical heads: ties across heads
     n = T - w
     _alloc_case(oracle, N, P, T, w, U, [0, 1, 12345, N * n // 3, N * n - 1, N * n], L=3)
+
+
+def test_three_quad_scorer_variant_in_a_subprocess(oracle):
+    """LUKV_QUADS=3 selects the scorer with three epilogue quads (read once per process, hence the
+    subprocess); it must meet the same tolerance and repeat bit for bit."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = f"""
+import sys
+sys.path.insert(0, {root!r}); sys.path.insert(0, {os.path.join(root, 'tests')!r})
+import numpy as np, torch
+from paper_2602_08585_b200 import lukv, synth
+from oracle import lukv_oracle
+from gpu_helpers import params_of, gpu_score, assert_scores_close, bits
+wl = synth.scaled(synth.CONFIGS["llama8b_1layer_8k"], L=2, H=3, T=6000 + 32, P=2, needles=16)
+q, k, _ = synth.gen_tensors(wl, "cuda")
+p = params_of(wl)
+a = gpu_score(p, q, k)
+b = gpu_score(p, q, k)
+assert torch.equal(a, b)
+ref = lukv_oracle.score(bits(q), bits(k), wl.G, wl.kp)
+assert_scores_close(a.cpu().numpy(), ref)
+print("ok")
+"""
+    env = dict(os.environ, LUKV_QUADS="3")
+    out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
