@@ -15,7 +15,9 @@
 // Work item = (head, run of item_tiles key tiles).  Items are dealt round-robin to a grid of
 // at most one CTA per SM, launched cooperatively (all CTAs resident).  A CTA runs pass 1
 // lag-1 items ahead of pass 2, so that the log-sum-exp of a head is normally complete before
-// pass 2 needs it, and the key tiles pass 2 re-reads are still in L2: K crosses HBM once.
+// pass 2 needs it.  With small items the key tiles pass 2 re-reads are still in L2 (K crosses
+// HBM once); the launcher prefers large items where there are enough of them, which re-read K
+// from HBM but change jobs less often (the kernel is bound by the exp2 evaluation, not by HBM).
 //
 // Warp roles per CTA: 4*NQ epilogue warps in NQ quads (a warp may only read the TMEM lanes
 // 32*(warp%4)..+31), then one warp each: TMA producer, MMA issuer 0 and TMEM owner, MMA issuer 1,
@@ -230,6 +232,9 @@ __device__ __forceinline__ uint64_t ex2_pair(uint64_t x) {
   unpack2(x, a, b);
   return pack2(ex2(a), ex2(b));
 }
+// Which exp2 pairs of a 32-element chunk go to the FMA pipe instead of the special-function unit (i is the
+// index of the group of four elements): one pair in eight in both passes, the measured optimum (one in
+// four already costs more issue slots and FMA-pipe time than the special-function unit gains).
 #ifndef LUKV_POLY_SEL1
 #define LUKV_POLY_SEL1(i) ((((i) >> 2) & 3) == 0)
 #endif
