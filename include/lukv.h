@@ -52,7 +52,8 @@ typedef enum lukv_status {
   LUKV_OK = 0,
   LUKV_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, flags != 0           */
   LUKV_ERR_UNSUPPORTED = -2,         /* d not in {64,128}, unknown dtype, even kp, (P-1) does  */
-                                     /* not divide T, G*w > 256, P > 4097, sizes beyond int32  */
+                                     /* not divide T, G*w > 256, P > 4097, N > 18944, sizes    */
+                                     /* beyond int32                                           */
   LUKV_ERR_BUDGET = -3,              /* some B_q < 0 or B_q > N*n; a ratio outside its range   */
   LUKV_ERR_WORKSPACE_TOO_SMALL = -4, /* ws_bytes < lukv_workspace_bytes()                      */
   LUKV_ERR_OUTPUT_TOO_SMALL = -5,    /* rows_cap < sum_q B_q + S*N*w                           */
@@ -66,7 +67,8 @@ enum { LUKV_DTYPE_BF16 = 0, LUKV_DTYPE_FP32 = 1 };
 typedef struct lukv_params {
   int32_t batch;        /* S >= 1                                                             */
   int32_t n_layers;     /* L >= 1                                                             */
-  int32_t n_kv_heads;   /* H >= 1                                                             */
+  int32_t n_kv_heads;   /* H >= 1, N = L*H <= 18944 (the greedy keeps 12 bytes of shared      */
+                        /* memory per head of a sequence)                                     */
   int32_t gqa_group;    /* G >= 1, G*w <= 256                                                 */
   int32_t head_dim;     /* d in {64, 128}                                                     */
   int32_t ctx_len;      /* T                                                                  */
@@ -165,7 +167,10 @@ LUKV_API int lukv_select_gather(const lukv_params_t* params, const float* scores
  * The allocation kernels run on an auxiliary stream beside the scorer; that stream and two
  * events are created on the first call on a device and kept until the process exits.  The
  * caller's stream waits for them inside the call, so everything the call enqueues is ordered
- * after earlier work on `stream` and before later work on it.
+ * after earlier work on `stream` and before later work on it.  Host threads may call
+ * concurrently on one device (each with its own workspace and outputs): the call holds a
+ * per-device lock while it enqueues on the auxiliary stream, so such calls enqueue one after
+ * the other.
  */
 LUKV_API int lukv_compress(const lukv_params_t* params, const void* q_win, const void* k, const void* v,
                   const float* curves, const int64_t* budgets_in, void* k_out, void* v_out, int32_t* kept_idx,

@@ -124,8 +124,8 @@ __device__ __forceinline__ long long capsum(int c, int seg, int n, int floor_tok
   return t > 0 ? t : 0;
 }
 
-// Block-wide sum; every thread gets the result.  `buf` holds one value per warp; two buffers are
-// used alternately so that one barrier per call is enough.
+// Block-wide sum; every thread gets the result.  `buf` holds one value per warp.  One barrier per
+// call is enough only if consecutive calls use different buffers: the caller alternates between two.
 __device__ __forceinline__ long long block_sum_ll(long long v, long long* buf) {
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
@@ -180,6 +180,7 @@ __global__ void __launch_bounds__(kGreedyMaxThreads) greedy_kernel(const float* 
     // them would change nothing
     int idx_bits = 0;
     while (idx_bits < 32 && ((unsigned long long)N * (unsigned)G1) >> idx_bits) ++idx_bits;
+    int round = 0;  // executed iterations: selects the sum buffer (the skipped bits must not count)
     for (int bit = 63; bit >= 0; --bit) {
       if (bit < 32 && bit >= idx_bits) continue;
       long long local = 0;
@@ -205,7 +206,7 @@ __global__ void __launch_bounds__(kGreedyMaxThreads) greedy_kernel(const float* 
         mid[h] = m;
         local += capsum(m, seg, n, floor_tok) - capsum(l, seg, n, floor_tok);
       }
-      const long long tokens0 = block_sum_ll(local, sum_buf[bit & 1]);
+      const long long tokens0 = block_sum_ll(local, sum_buf[round++ & 1]);
       if (tokens0 > R) {
         for (int h = tid; h < N; h += nthr) hi[h] = mid[h];
       } else {

@@ -54,6 +54,8 @@ static int make_dims(const lukv_params_t* p, Dims* dm) {
   if (p->ctx_len % (p->curve_points - 1) != 0) return LUKV_ERR_UNSUPPORTED;
   if ((int64_t)p->gqa_group * p->window > 256) return LUKV_ERR_UNSUPPORTED;
   const int64_t N = (int64_t)p->n_layers * p->n_kv_heads;
+  // the greedy kernel keeps three 32-bit indices per head in the shared memory of one CTA
+  if (N > kGreedyMaxHeads) return LUKV_ERR_UNSUPPORTED;
   const int64_t heads = N * p->batch;
   // packed row indices, segment ids k*N+hid and grid sizes must fit 32 bits
   if (heads * p->ctx_len >= (int64_t)1 << 31 || N * (p->curve_points - 1) >= (int64_t)1 << 31 || heads > (1 << 24))
@@ -116,6 +118,9 @@ struct SideStream {
   cudaStream_t stream = nullptr;
   cudaEvent_t fork = nullptr, join = nullptr;
   bool ok = false;
+  // held while a call records and waits on the two events: a second host thread that calls on the same
+  // device must not re-record them between this call's record and the wait that belongs to it
+  std::mutex use;
 };
 static SideStream* side_stream() {
   static SideStream table[64];
@@ -147,6 +152,7 @@ static int run_compress(const Dims& dm, const void* q_win, const void* k, const 
   SideStream* side = (overlap && tc) ? side_stream() : nullptr;
   int rc = LUKV_OK;
   if (side) {
+    std::lock_guard<std::mutex> in_use(side->use);
     LaunchCtx ls;
     ls.st = side->stream;
     if (cudaEventRecord(side->fork, lc.st) != cudaSuccess || cudaStreamWaitEvent(ls.st, side->fork, 0) != cudaSuccess)
@@ -286,7 +292,10 @@ int lukv_compress_profile(const lukv_params_t* params, const void* q_win, const 
   cudaEvent_t ev[65];
   const char* names[64];
   for (int i = 0; i <= max_times; ++i)
-    if (cudaEventCreate(&ev[i]) != cudaSuccess) return LUKV_ERR_CUDA;
+    if (cudaEventCreate(&ev[i]) != cudaSuccess) {
+      while (--i >= 0) cudaEventDestroy(ev[i]);
+      return LUKV_ERR_CUDA;
+    }
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;
   lc.events = ev;

@@ -42,6 +42,10 @@ size_t score_tc_stats_bytes(const Dims& dm);            // pass-1 partials of th
 size_t score_tc_flag_bytes(const Dims& dm);             // its zero-initialised counters and (lse, tag) rows
 Workspace carve_workspace(const Dims& dm, void* base);  // base may be null (size query)
 
+// Heads per sequence the greedy kernel can hold: 12 bytes of shared memory each, 227 KB per CTA
+// less its static arrays.
+constexpr int kGreedyMaxHeads = 18944;
+
 // Launch bookkeeping: counts the kernels a call enqueues and, when a timeline is attached
 // (profiling entry point only), records a CUDA event after each of them.
 struct LaunchCtx {

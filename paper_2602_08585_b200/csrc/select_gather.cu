@@ -1,7 +1,7 @@
 // Stages (c) and (d): per-head variable-k top-k selection and the packed gather.
-//   select_kernel  one CTA per head: the b-th largest score is found by a bit-by-bit
-//                  search over the order-preserving integer image of the scores
-//                  (32 block-wide counts), then the kept positions are emitted in
+//   select_kernel  one CTA per head: the b-th largest score is found digit by digit (11, 11
+//                  and 10 bits) over the order-preserving integer image of the scores, each
+//                  digit from a shared-memory histogram, then the kept positions are emitted in
 //                  ascending order: everything above the threshold plus the first
 //                  (lowest-position) ties.  This realises M^pi(b) of Sec. 3.2 / the
 //                  "Eviction" step of Sec. 4.3 without a full sort.
@@ -254,6 +254,9 @@ template <int LPR>
 void launch_gather_t(const Dims& dm, const int32_t* offsets, const int32_t* kept_idx, const void* k, const void* v,
                      void* k_out, void* v_out, long long rows_cap, HeadRange hr, cudaStream_t st) {
   // the rows of a head range are only known on the device; size the grid for its share of the output
+  // (a capacity beyond what the call can ever produce sizes nothing: clamp it first)
+  const long long rows_max = (long long)dm.heads() * dm.T;
+  if (rows_cap > rows_max) rows_cap = rows_max;
   const long long spans = (rows_cap * hr.nh / (long long)dm.heads() + 31) / 32 + 1;
   long long blocks = (spans + kGatherThreads / 32 - 1) / (kGatherThreads / 32);
   const long long max_blocks = 148LL * 8 * 4;  // a few waves of resident CTAs; the loop covers the rest

@@ -41,6 +41,10 @@ def _p(**kw):
     return lukv.make_params(**base)
 
 
+def test_largest_head_count_is_accepted():
+    assert lukv.lukv_workspace_bytes(_p(L=18944, H=1)) > 0
+
+
 def test_workspace_bytes_grows_with_the_problem():
     a = lukv.lukv_workspace_bytes(_p())
     b = lukv.lukv_workspace_bytes(_p(T=512))
@@ -51,6 +55,7 @@ def test_workspace_bytes_grows_with_the_problem():
 @pytest.mark.parametrize("kw,code", [
     (dict(d=96), lukv.ERR_UNSUPPORTED), (dict(dtype=7), lukv.ERR_UNSUPPORTED), (dict(kp=4), lukv.ERR_UNSUPPORTED),
     (dict(P=18), lukv.ERR_UNSUPPORTED), (dict(G=64), lukv.ERR_UNSUPPORTED), (dict(P=8193, T=8192), lukv.ERR_UNSUPPORTED),
+    (dict(L=18945, H=1), lukv.ERR_UNSUPPORTED),   # heads per sequence beyond the greedy kernel's shared memory
     (dict(w=256), lukv.ERR_INVALID_ARG), (dict(w=0), lukv.ERR_INVALID_ARG), (dict(S=0), lukv.ERR_INVALID_ARG),
     (dict(P=1), lukv.ERR_INVALID_ARG), (dict(kp=0), lukv.ERR_INVALID_ARG), (dict(scale=-1.0), lukv.ERR_INVALID_ARG),
 ])

@@ -1,4 +1,4 @@
-"""The workspace-free allocation entry point against the regular one.
+"""The workspace-free allocation entry point against the regular one and against the oracle.
 
 lukv_allocate_static serves callers that cannot allocate device memory when budgets are
 needed (for instance a server whose memory belongs to its own pool): its scratch is a fixed
@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import lukv_oracle
 from paper_2602_08585_b200 import lukv, synth
 from gpu_helpers import gpu_allocate
 
@@ -38,6 +39,9 @@ def test_static_allocate_matches_allocate_on_two_calls_in_a_row():
         np.testing.assert_array_equal(b_static, b_ref)          # integer outputs: bit-exact
         np.testing.assert_array_equal(o_static, o_ref)
         np.testing.assert_array_equal(b_static.sum(axis=1), wl.budgets())
+        b_orc, o_orc = lukv_oracle.allocate(curves, wl.T, wl.w, wl.budgets())
+        np.testing.assert_array_equal(b_static, b_orc)
+        np.testing.assert_array_equal(o_static, o_orc)
 
 
 def test_static_allocate_rejects_sizes_beyond_its_scratch():
