@@ -37,7 +37,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama8b_32k")
+    ap.add_argument("--workload", default="llama8b_32k",
+                    help="a configuration name, or 'all': one JSON line per configuration (single GPU)")
     ap.add_argument("--path", default="compress", choices=["compress", "profile"],
                     help="compress: the headline path; profile: the offline profile build and the online "
                          "lookup front end (secondary measurement, single GPU)")
@@ -109,13 +110,21 @@ def run_reference(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded)",
         "config": {"workload": wl.name, "S": wl.S, "heads": wl.N, "T": wl.T, "w": wl.w, "keep": list(wl.keep),
                    "n_sink": args.sinks, "min_keep": args.min_keep},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "host_cores": host_cores(), "kind": "oracle",
                          "sample": f"{heads} of {wl.S * wl.N} heads per step (score+select+gather) plus the full "
                                    "allocation, single thread, extrapolated to all heads"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+def host_cores() -> int:
+    """Cores this process may run on (the oracle itself uses one thread)."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
 
 
 # ---- clocks ------------------------------------------------------------------------------------
@@ -203,7 +212,7 @@ def kernel_bytes(name, wl, rows):
     score_bytes = heads * wl.n * 4
     row = wl.d * es
     if name.startswith("score") and "lse" not in name:
-        return k_bytes + q_bytes + (score_bytes if name.endswith("2") or "fused" in name else 0)
+        return k_bytes + q_bytes + (score_bytes if name.endswith("2") or "fused" in name or "onepass" in name else 0)
     if name == "max_pool":
         return 2 * score_bytes
     if name == "select":
@@ -304,25 +313,30 @@ def run_ours(args):
     dom_bytes = kernel_bytes(dom, wl, out.rows)
     dom_s = kernels[dom]["ms_per_launch"] * 1e-3
     dom_gbs = dom_bytes / dom_s / 1e9
-    if dom == "score_fused":
-        # The fused scorer evaluates one exp2 per (query row, visible key) in each of its two passes on the
-        # special-function units, which do 16 per clock and SM: that, not HBM, bounds it (K crosses HBM
-        # once; the second pass reads it from L2).  Peak = 16 x SMs x max SM clock.
-        import torch
+    # The bound of record is HBM: the path streams K once and copies the kept rows, and the scorer's algorithmic
+    # bytes are K + Q read and the raw scores written.  `frac` = algorithmic bytes / kernel time / measured copy peak.
+    roofline = {"kernel": dom, "bound": "hbm", "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
+                "frac": dom_gbs / peak, "frac_of_nominal_8TBs": dom_gbs / NOMINAL_HBM_GBS, "peak_source": peak_src,
+                "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_s * 1e3,
+                "traffic": load_traffic(dom, wl.name)}
+    if roofline["traffic"]:
+        roofline["traffic_gbs"] = roofline["traffic"] / dom_s / 1e9
+        roofline["traffic_over_algorithmic"] = roofline["traffic"] / dom_bytes
+    if dom.startswith("score") and wl.dtype == "bf16" and wl.d == 128:
+        # What holds the tensor-core scorer below the HBM bound: one exp2 per (query row, key) is the method's
+        # work; the two-sweep kernel evaluates every one twice (once for the row normaliser, once for the
+        # probability).  The unit rate is the special-function units' (16 per clock and SM).
         sms = torch.cuda.get_device_properties(local).multi_processor_count
-        exps = 2.0 * wl.S * wl.N * wl.G * wl.w * wl.T
+        exps = 1.0 * wl.S * wl.N * wl.G * wl.w * wl.T
+        sweeps = 1 if "onepass" in dom else 2
         peak_exp = 16.0 * sms * (sampler.max_mhz or 1965) * 1e6 / 1e9
-        roofline = {"kernel": dom, "bound": "alu", "achieved": exps / dom_s / 1e9, "peak": peak_exp,
-                    "unit": "Gexp2/s", "frac": exps / dom_s / 1e9 / peak_exp,
-                    "peak_source": "16 exp2 per clock per SM (special-function unit) x SM count x max SM clock; one exp2 pair in "
-                                   "eight is evaluated on the FMA pipe instead, so the ceiling is 8/7 of it",
-                    "algorithmic_exp2_per_launch": exps, "algorithmic_bytes_per_launch": dom_bytes,
-                    "hbm_achieved_gbs": dom_gbs, "hbm_peak_gbs": peak, "hbm_frac": dom_gbs / peak,
-                    "hbm_peak_source": peak_src, "traffic": load_traffic(dom, wl.name)}
-    else:
-        roofline = {"kernel": dom, "bound": "hbm", "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
-                    "frac": dom_gbs / peak, "peak_source": peak_src, "algorithmic_bytes_per_launch": dom_bytes,
-                    "traffic": load_traffic(dom, wl.name)}
+        roofline["exp2"] = {"algorithmic_exp2_per_launch": exps, "evaluated_exp2_per_launch": sweeps * exps,
+                            "achieved_gexp2_s": exps / dom_s / 1e9,
+                            "evaluated_gexp2_s": sweeps * exps / dom_s / 1e9,
+                            "unit_peak_gexp2_s": peak_exp, "frac_of_unit_peak_on_algorithmic": exps / dom_s / 1e9 / peak_exp,
+                            "frac_of_unit_peak_on_evaluated": sweeps * exps / dom_s / 1e9 / peak_exp,
+                            "unit_peak_source": "16 exp2 per clock per SM x SM count x max SM clock; the rates the "
+                                                "epilogue reaches in isolation are in profiles/exp2_epilogue_rates.md"}
     es = 2 if wl.dtype == "bf16" else 4
     path_bytes = wl.S * wl.N * wl.T * wl.d * es + 2 * out.rows * wl.d * es   # K read + kept K/V written
     path_gbs = path_bytes / (ms * 1e-3) / 1e9
@@ -421,7 +435,8 @@ def run_ours(args):
         from oracle import lukv_oracle as O
         O.build()
         sec, extrap, used = oracle_sample_seconds(wl, args.cpu_heads, args.sinks, args.min_keep)
-        cpu_baseline = {"value": wl.S * wl.T / extrap, "unit": UNIT, "cores": 1, "kind": "oracle",
+        cpu_baseline = {"value": wl.S * wl.T / extrap, "unit": UNIT, "cores": 1, "host_cores": host_cores(),
+                        "kind": "oracle",
                         "seconds_for_sample": sec,
                         "sample": f"{used} of {wl.S * wl.N} heads (score+select+gather) plus the full allocation, "
                                   "single thread, extrapolated to all heads"}
@@ -545,7 +560,8 @@ def run_profile_path(args):
         t0 = time.perf_counter()
         O.profile_build(U_np[:6], Tc, wl.w, ratios)
         sec = time.perf_counter() - t0
-        cpu = {"value": 6 * R / sec, "unit": "(query, ratio) allocations/s", "cores": 1, "kind": "oracle",
+        cpu = {"value": 6 * R / sec, "unit": "(query, ratio) allocations/s", "cores": 1, "host_cores": host_cores(),
+               "kind": "oracle",
                "seconds_for_sample": sec, "sample": f"6 of {Mq} calibration queries, all {R} ratios, single thread"}
     es = 2 if wl.dtype == "bf16" else 4
     print(json.dumps({
@@ -583,6 +599,21 @@ def main():
     elif args.path == "profile":
         if int(os.environ.get("RANK", "0")) == 0:
             run_profile_path(args)
+    elif args.workload == "all":
+        # one line per configuration, each with its own roofline and clocks (single GPU; the end-to-end and CPU
+        # legs only for the headline configuration)
+        from paper_2602_08585_b200 import synth
+        assert int(os.environ.get("WORLD_SIZE", "1")) == 1, "--workload all is a single-GPU run"
+        for name in synth.CONFIGS:
+            sub = argparse.Namespace(**vars(args))
+            sub.workload = name
+            if name != "llama8b_32k":
+                sub.no_e2e = sub.no_cpu_baseline = True
+            run_ours(sub)
+            import gc
+            import torch
+            gc.collect()
+            torch.cuda.empty_cache()
     else:
         run_ours(args)
 

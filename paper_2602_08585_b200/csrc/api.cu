@@ -26,8 +26,10 @@ Workspace carve_workspace(const Dims& dm, void* base) {
   ws.raw = static_cast<float*>(take(heads * dm.n * sizeof(float)));
   ws.pooled = static_cast<float*>(take(heads * dm.n * sizeof(float)));
   const size_t stats_simt = heads * score_chunks(dm) * dm.M * 2 * sizeof(float);
-  const size_t stats_tc = score_tc_stats_bytes(dm);
-  ws.stats = static_cast<float*>(take(stats_simt > stats_tc ? stats_simt : stats_tc));
+  size_t stats_bytes = score_tc_stats_bytes(dm);
+  if (stats_simt > stats_bytes) stats_bytes = stats_simt;
+  if (score_onepass_stats_bytes(dm) > stats_bytes) stats_bytes = score_onepass_stats_bytes(dm);
+  ws.stats = static_cast<float*>(take(stats_bytes));
   ws.lse = static_cast<float*>(take(heads * dm.M * sizeof(float)));
   ws.gains = static_cast<float*>(take((size_t)dm.N * (dm.P - 1) * sizeof(float)));
   ws.head_flags = static_cast<int*>(take(score_tc_flag_bytes(dm)));

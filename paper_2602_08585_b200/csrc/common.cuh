@@ -38,8 +38,14 @@ struct Workspace {
 };
 
 int score_chunks(const Dims& dm);                       // key chunks per head of the SIMT scorer
-size_t score_tc_stats_bytes(const Dims& dm);            // pass-1 partials of the tensor-core scorer
-size_t score_tc_flag_bytes(const Dims& dm);             // its zero-initialised counters and (lse, tag) rows
+size_t score_tc_stats_bytes(const Dims& dm);            // pass-1 partials of the two-sweep tensor-core scorer
+size_t score_tc_flag_bytes(const Dims& dm);             // zero-initialised block: [heads] counters, then the (lse, tag) rows
+size_t score_tc_lse_offset(const Dims& dm);             // offset of the (lse, tag) rows inside that block
+void score_test_hooks(uint32_t* spin_limit, int* drop_item);  // environment hooks for the timeout tests
+// Single-sweep tensor-core scorer: takes a shape if a head's work items fit kOnePassMaxItems CTAs.
+constexpr int kOnePassMaxItems = 128;
+bool score_onepass_eligible(const Dims& dm);
+size_t score_onepass_stats_bytes(const Dims& dm);       // its per-(row, key tile) partials; 0 if not eligible
 Workspace carve_workspace(const Dims& dm, void* base);  // base may be null (size query)
 
 // Heads per sequence the greedy kernel can hold: 12 bytes of shared memory each, 227 KB per CTA
@@ -78,6 +84,9 @@ bool score_tc_supported(const Dims& dm);
 // spare_sms: SMs the persistent grid leaves to kernels of other streams
 cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const Workspace& ws, int32_t* dev_status,
                             HeadRange hr, bool clear_flags, int spare_sms, LaunchCtx& lc);
+// The single-sweep kernel alone; cudaErrorNotSupported (nothing launched) if the device has too few SMs for the shape.
+cudaError_t launch_score_onepass(const Dims& dm, const void* q, const void* k, const Workspace& ws,
+                                 int32_t* dev_status, HeadRange hr, bool clear_flags, int spare_sms, LaunchCtx& lc);
 cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, HeadRange hr, LaunchCtx& lc);
 cudaError_t launch_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, float* gains,
                             int32_t* budgets, int32_t* offsets, LaunchCtx& lc);

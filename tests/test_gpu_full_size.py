@@ -69,7 +69,14 @@ def _check_full(oracle, name, sample_heads):
 
     # ---- sampled heads against the oracle
     rng = np.random.default_rng(wl.seed)
-    sample = sorted(set(int(x) for x in rng.integers(0, heads, size=sample_heads)) | {0, heads - 1})
+    sample = set(int(x) for x in rng.integers(0, heads, size=sample_heads)) | {0, heads - 1}
+    if wl.S > 1:
+        # mixed budgets: the same number of heads from every sequence parity (the keep fractions alternate)
+        per_kind = (sample_heads + 1) // 2
+        for parity in (0, 1):
+            seqs = rng.choice(np.arange(parity, wl.S, 2), size=per_kind)
+            sample |= set(int(sq) * wl.N + int(h) for sq, h in zip(seqs, rng.integers(0, wl.N, size=per_kind)))
+    sample = sorted(sample)
     kept_np = out.kept_idx.cpu().numpy()
     agree = total = 0
     for u in sample:
@@ -98,15 +105,15 @@ def _check_full(oracle, name, sample_heads):
 
 
 def test_llama8b_32k_full(oracle):
-    _check_full(oracle, "llama8b_32k", sample_heads=6)
+    _check_full(oracle, "llama8b_32k", sample_heads=32)
 
 
 def test_batch8_16k_mixed_full(oracle):
-    _check_full(oracle, "batch8_16k_mixed", sample_heads=6)
+    _check_full(oracle, "batch8_16k_mixed", sample_heads=16)
 
 
 def test_gqa7_128k_full(oracle):
-    _check_full(oracle, "gqa7_128k", sample_heads=2)
+    _check_full(oracle, "gqa7_128k", sample_heads=8)
 
 
 def test_repeated_calls_are_bit_identical():
