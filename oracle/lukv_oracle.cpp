@@ -22,6 +22,10 @@
 //   gather   : the retained index set I of Sec. 3.2 materialised as a packed cache.
 //   curves   : utility-versus-budget curve of a proxy metric = running sum of the oracle
 //              importance in the metric's ranking order (Sec. 3.2, Eq. "head_loss_def").
+//   importance : the oracle importance of Sec. 4.1 (Eq. "oracle_importance"): the largest contribution
+//              a cached position makes to the head output over K_max decode steps, attention weight
+//              times the L2 norm of the projected value (App. E names the norm and an intra-layer
+//              normalisation); readings for grouped queries and the normalisation in the design notes.
 //   exact    : the allocation problem on the raw curves by the multiple-choice-knapsack
 //              recursion (Sec. 4.2 mentions the exact solver as the comparison point).
 //   deployment settings (App. E): attention sinks always ranked first; a minimum number of
@@ -39,7 +43,10 @@
 // points rho = 0 and 1, budget conservation and monotonicity in rho; lookup against a
 // hand-worked example; curves against the pinned selection (importance mass of M^pi(k)), a
 // library sort for the oracle metric, and closed forms; the exact solver against exhaustive
-// search, against the greedy on concave curves, and between the greedy's raw and hull values.
+// search, against the greedy on concave curves, and between the greedy's raw and hull values;
+// the oracle importance against a library softmax times a library vector norm (one decode step,
+// identity projection), closed forms for identical keys, monotonicity in K_max, a dominant decode
+// key, doubling under two identical grouped query heads, and unit mass per layer after normalisation.
 // No function here is "parity unpinned".
 //
 // Build: g++ -O2 -std=c++17 -ffp-contract=off -shared -fPIC lukv_oracle.cpp -o liblukv_oracle.so
@@ -449,6 +456,82 @@ int oracle_exact_allocate(const float* curves, int N, int P, int T, int w, int S
   }
   return 0;
 }
+
+// Oracle importance (Sec. 4.1, Eq. "oracle_importance"):  I_j = max_{k=1..K_max} A_{k,j} * || v_j W_O ||_2.
+//   A_{k,j}: attention weight (Eq. 1) of the query of decode step k on cached position j.  The softmax of step k
+//            runs over the T cached positions and, when decode keys are given, over the keys of decode steps
+//            1..k as well (causal, the step's own key included).
+//   grouped queries: a KV head is read by G query heads, each with its own slice of the output projection;
+//            the importance of a cached position adds their contributions before the maximum over the steps:
+//            I_j = max_k sum_g A_{g,k,j} * || v_j W_O^(g) ||_2   (G = 1 is the paper's formula as printed).
+//   normalisation (App. E, "intra-layer normalisation"): every layer's values are divided by their sum over the
+//            layer's heads and rankable positions, so that each layer carries unit mass.
+// q_dec [S][L][H*G][Kmax][d], k, v [S][L][H][T][d], k_dec [S][L][H][Kmax][d] or null, w_o [L][H*G][d][Dm];
+// out importance [S][L*H][T-w] fp32 (window positions are always kept and never enter a loss).
+void oracle_importance(const void* q_dec, const void* k, const void* v, const void* k_dec, const void* w_o, int dtype,
+                       int S, int L, int H, int G, int d, int T, int w, int Kmax, int Dm, float scale_in,
+                       int normalize, float* importance) {
+  const int n = T - w;
+  const double scale = scale_in > 0.f ? static_cast<double>(scale_in) : 1.0 / std::sqrt(static_cast<double>(d));
+  std::vector<double> imp(static_cast<size_t>(S) * L * H * n);
+  std::vector<double> vnorm(static_cast<size_t>(G) * T), x(static_cast<size_t>(T) + Kmax), s(T), y(Dm);
+  for (int q = 0; q < S; ++q)
+    for (int l = 0; l < L; ++l)
+      for (int h = 0; h < H; ++h) {
+        const int64_t u = (static_cast<int64_t>(q) * L + l) * H + h;
+        const int64_t kbase = u * T * d, dbase = u * Kmax * d;
+        // || v_j W_O^(g) ||_2
+        for (int g = 0; g < G; ++g) {
+          const int64_t wbase = (static_cast<int64_t>(l) * H * G + h * G + g) * d * Dm;
+          for (int j = 0; j < T; ++j) {
+            std::fill(y.begin(), y.end(), 0.0);
+            for (int c = 0; c < d; ++c) {
+              const double vc = load_elem(v, dtype, kbase + static_cast<int64_t>(j) * d + c);
+              for (int m = 0; m < Dm; ++m) y[m] += vc * load_elem(w_o, dtype, wbase + static_cast<int64_t>(c) * Dm + m);
+            }
+            double ss = 0.0;
+            for (int m = 0; m < Dm; ++m) ss += y[m] * y[m];
+            vnorm[static_cast<size_t>(g) * T + j] = std::sqrt(ss);
+          }
+        }
+        double* out = imp.data() + u * n;
+        std::fill(out, out + n, 0.0);
+        for (int kk = 0; kk < Kmax; ++kk) {
+          std::fill(s.begin(), s.end(), 0.0);
+          for (int g = 0; g < G; ++g) {
+            const int64_t qbase = (((static_cast<int64_t>(q) * L + l) * H * G + h * G + g) * Kmax + kk) * d;
+            const int visible = T + (k_dec ? kk + 1 : 0);
+            double mx = -std::numeric_limits<double>::infinity();
+            for (int j = 0; j < visible; ++j) {
+              double dot = 0.0;
+              for (int c = 0; c < d; ++c) {
+                const double kc = j < T ? load_elem(k, dtype, kbase + static_cast<int64_t>(j) * d + c)
+                                        : load_elem(k_dec, dtype, dbase + static_cast<int64_t>(j - T) * d + c);
+                dot += load_elem(q_dec, dtype, qbase + c) * kc;
+              }
+              x[j] = dot * scale;
+              mx = std::max(mx, x[j]);
+            }
+            double Z = 0.0;
+            for (int j = 0; j < visible; ++j) Z += std::exp(x[j] - mx);
+            for (int j = 0; j < T; ++j) s[j] += std::exp(x[j] - mx) / Z * vnorm[static_cast<size_t>(g) * T + j];
+          }
+          for (int j = 0; j < n; ++j) out[j] = std::max(out[j], s[j]);
+        }
+      }
+  if (normalize) {
+    for (int q = 0; q < S; ++q)
+      for (int l = 0; l < L; ++l) {
+        double* base = imp.data() + (static_cast<int64_t>(q) * L + l) * H * n;
+        double total = 0.0;
+        for (int64_t i = 0; i < static_cast<int64_t>(H) * n; ++i) total += base[i];
+        if (total > 0.0)
+          for (int64_t i = 0; i < static_cast<int64_t>(H) * n; ++i) base[i] /= total;
+      }
+  }
+  for (size_t i = 0; i < imp.size(); ++i) importance[i] = to_f32_ftz(imp[i]);
+}
+
 
 // Utility-versus-budget curves of a proxy metric (Sec. 3.2: M^pi(k) is the set of the first k
 // positions when ranked by pi; Eq. "head_loss_def": the eviction loss of a retained set is the

@@ -228,6 +228,22 @@ def build_curves(scores, importance, T: int, w: int, P: int, n_sink: int = 0) ->
     return curves
 
 
+def importance(q_dec, k, v, w_o, G: int, w: int, k_dec=None, scale: float = 0.0, normalize: bool = True) -> np.ndarray:
+    """Oracle importance (Sec. 4.1): q_dec [S][L][H*G][Kmax][d], k, v [S][L][H][T][d], w_o [L][H*G][d][Dm],
+    k_dec [S][L][H][Kmax][d] or None -> importance [S][L*H][T-w] float32."""
+    q_dec, k, v, w_o = _c(q_dec), _c(k), _c(v), _c(w_o)
+    k_dec = None if k_dec is None else _c(k_dec)
+    S, L, HG, Kmax, d = q_dec.shape
+    H, T = k.shape[2], k.shape[3]
+    Dm = w_o.shape[3]
+    assert HG == H * G and v.shape == k.shape and w_o.shape == (L, H * G, d, Dm)
+    assert k_dec is None or k_dec.shape == (S, L, H, Kmax, d)
+    out = np.empty((S, L * H, T - w), np.float32)
+    lib().oracle_importance(_p(q_dec), _p(k), _p(v), _p(k_dec), _p(w_o), _dtype_code(k), S, L, H, G, d, T, w, Kmax, Dm,
+                            ctypes.c_float(scale), int(bool(normalize)), _p(out))
+    return out
+
+
 def exact_allocate(curves, T: int, w: int, budgets_in):
     """Exact allocation on token-resolution curves [N][T+1] -> (budgets [S][N] int32, optimum values [S] float64)."""
     curves = _c(curves, np.float32)
