@@ -274,8 +274,8 @@ LUKV_API int lukv_profile_budgets(const lukv_params_t* params, const float* prof
  * The ranking is the selection's (sinks first, score descending, lower position first among
  * equals).  Sums are fp64 in ranking order, each point rounded once to fp32.  With S calibration
  * queries as the batch, the output is the [n_queries][N][P] input of lukv_profile_build.
- * The oracle importance itself (Eq. "oracle_importance") needs the model's decoding run and is an
- * input here.
+ * The oracle importance (Eq. "oracle_importance") is an input here; lukv_oracle_importance computes it from
+ * decode queries, the cache and the output projection.
  *
  *   scores      [S][N][n] fp32   proxy scores of the rankable positions (lukv_score)
  *   importance  [S][N][n] fp32   oracle importance of the same positions
@@ -286,6 +286,36 @@ LUKV_API int lukv_profile_budgets(const lukv_params_t* params, const float* prof
  */
 LUKV_API int lukv_build_curves(const lukv_params_t* params, const float* scores, const float* importance,
                                float* curves, void* stream);
+
+/*
+ * Oracle importance (Sec. 4.1, Eq. "oracle_importance"): the largest contribution a cached position makes to
+ * the head output over K_max future decode steps,
+ *     I_j = max_{k = 1..K_max}  A_{k,j} * || v_j W_O ||_2 ,
+ * A_{k,j} being the attention weight (Eq. 1) of the query of decode step k on cached position j and W_O the
+ * head's slice of the output projection; App. E names the L2 norm and an intra-layer normalisation.  An offline
+ * analysis tool: its output, with the proxy scores of the same context, is the input of lukv_build_curves.
+ * Where the paper leaves a choice:
+ *   - the softmax of step k runs over the T cached positions and, if k_dec is given, over the keys of decode
+ *     steps 1..k as well (the step's own key included); k_dec = NULL restricts it to the cached positions;
+ *   - a KV head is read by G query heads, each with its own slice of W_O: their contributions are added before
+ *     the maximum over the steps, I_j = max_k sum_g A_{g,k,j} * || v_j W_O^(g) ||_2 (G = 1: the formula above);
+ *   - normalize != 0: every layer's values are divided by their sum over the layer's H heads and n rankable
+ *     positions (fp64 total), so each layer of each sequence carries unit mass; 0 leaves them as they are.
+ * Window positions are always kept and get no value: the output covers the n = T-w rankable positions.
+ *
+ *   q_dec       [S][L][H*G][k_max][d]   queries of the k_max decode steps (query head h*G+g reads KV head h)
+ *   k, v        [S][L][H][T][d]         the prefill cache
+ *   k_dec       [S][L][H][k_max][d]     keys of the decode steps, or NULL
+ *   w_o         [L][H*G][d][d_model]    output projection, one [d][d_model] slice per query head, in the
+ *                                       element type of the cache
+ *   importance  [S][N][n] fp32          out
+ *   ws          lukv_importance_workspace_bytes() bytes, 256-byte aligned (value norms and row log-sum-exps)
+ * fp32 arithmetic on the inputs as given; params->pool_kernel and curve_points must be valid but are unused.
+ */
+LUKV_API int lukv_importance_workspace_bytes(const lukv_params_t* params, int32_t k_max, size_t* bytes /* HOST, out */);
+LUKV_API int lukv_oracle_importance(const lukv_params_t* params, int32_t k_max, int32_t d_model, const void* q_dec,
+                                    const void* k, const void* v, const void* k_dec, const void* w_o,
+                                    int32_t normalize, float* importance, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Exact allocation (Sec. 4.2, Eq. "combinatorial_optimization": maximise the summed utility over

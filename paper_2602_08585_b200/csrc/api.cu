@@ -493,6 +493,38 @@ int lukv_build_curves(const lukv_params_t* params, const float* scores, const fl
   return LUKV_OK;
 }
 
+int lukv_importance_workspace_bytes(const lukv_params_t* params, int32_t k_max, size_t* bytes) {
+  Dims dm;
+  if (!bytes || k_max < 1) return LUKV_ERR_INVALID_ARG;
+  const int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if ((int64_t)dm.heads() * dm.G * k_max >= (int64_t)1 << 31) return LUKV_ERR_UNSUPPORTED;
+  *bytes = importance_workspace_bytes(dm, k_max);
+  return LUKV_OK;
+}
+
+int lukv_oracle_importance(const lukv_params_t* params, int32_t k_max, int32_t d_model, const void* q_dec,
+                           const void* k, const void* v, const void* k_dec, const void* w_o, int32_t normalize,
+                           float* importance, void* ws, size_t ws_bytes, void* stream) {
+  Dims dm;
+  int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (k_max < 1 || d_model < 1 || !q_dec || !k || !v || !w_o || !importance || !ws ||
+      (reinterpret_cast<uintptr_t>(ws) & 255u) || !aligned16(q_dec) || !aligned16(k) || !aligned16(v) ||
+      (k_dec && !aligned16(k_dec)))
+    return LUKV_ERR_INVALID_ARG;
+  // grid dimensions: (heads * G) in x, tiles of 64 positions or blocks of 16 steps in y
+  if ((int64_t)dm.heads() * dm.G * k_max >= (int64_t)1 << 31 || (dm.n + 63) / 64 > 65535 || (k_max + 15) / 16 > 65535)
+    return LUKV_ERR_UNSUPPORTED;
+  if (ws_bytes < importance_workspace_bytes(dm, k_max)) return LUKV_ERR_WORKSPACE_TOO_SMALL;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  if (launch_importance(dm, k_max, d_model, q_dec, k, v, k_dec, w_o, normalize != 0, importance, ws, lc) != cudaSuccess)
+    return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
+}
+
 // Token resolution, no minimum retention: what the exact solver covers.
 static int make_exact_dims(const lukv_params_t* params, Dims* dm) {
   const int rc = make_dims(params, dm);

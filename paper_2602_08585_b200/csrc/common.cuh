@@ -107,6 +107,11 @@ cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, cons
 size_t curves_smem_bytes(int n, int P);
 cudaError_t launch_build_curves(const Dims& dm, const float* scores, const float* importance, float* curves,
                                 LaunchCtx& lc);
+// Oracle importance of Sec. 4.1 from decode queries, the cache and the output projection.
+size_t importance_workspace_bytes(const Dims& dm, int k_max);
+cudaError_t launch_importance(const Dims& dm, int k_max, int d_model, const void* q_dec, const void* k, const void* v,
+                              const void* k_dec, const void* w_o, bool normalize, float* importance, void* ws,
+                              LaunchCtx& lc);
 // Exact allocation (dynamic programme over the heads) at token resolution.
 size_t exact_workspace_bytes(const Dims& dm, int64_t max_budget);
 cudaError_t launch_exact_allocate(const Dims& dm, const float* curves, const int64_t* budgets_host, int32_t* budgets,

@@ -23,7 +23,7 @@ DTYPE_BF16, DTYPE_FP32 = 0, 1
 EXPORTS = ("lukv_workspace_bytes", "lukv_score", "lukv_allocate", "lukv_select_gather", "lukv_compress",
            "lukv_strerror", "lukv_last_launch_count", "lukv_compress_profile", "lukv_allocate_static",
            "lukv_profile_workspace_bytes", "lukv_profile_build", "lukv_profile_budgets", "lukv_build_curves", "lukv_exact_workspace_bytes",
-           "lukv_exact_allocate")
+           "lukv_exact_allocate", "lukv_importance_workspace_bytes", "lukv_oracle_importance")
 
 
 class Params(ctypes.Structure):
@@ -81,6 +81,9 @@ def lib() -> ctypes.CDLL:
         L.lukv_build_curves.argtypes = [pp, vp, vp, vp, vp]
         L.lukv_exact_workspace_bytes.argtypes = [pp, i64, ctypes.POINTER(sz)]
         L.lukv_exact_allocate.argtypes = [pp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.lukv_importance_workspace_bytes.argtypes = [pp, ctypes.c_int32, ctypes.POINTER(sz)]
+        L.lukv_oracle_importance.argtypes = [pp, ctypes.c_int32, ctypes.c_int32, vp, vp, vp, vp, vp, ctypes.c_int32, vp,
+                                             vp, sz, vp]
         L.lukv_strerror.argtypes = [ctypes.c_int]
         L.lukv_strerror.restype = ctypes.c_char_p
         for name in EXPORTS[:5] + EXPORTS[6:]:
@@ -196,6 +199,24 @@ def lukv_build_curves(params: Params, scores, importance, curves, stream=None, c
     """Curves of the proxy ranking: scores, importance [S][N][n] -> curves [S][N][P] (all device)."""
     rc = lib().lukv_build_curves(ctypes.byref(params), _ptr(scores), _ptr(importance), _ptr(curves), _stream(stream))
     return _check(rc, "lukv_build_curves", check)
+
+
+def lukv_importance_workspace_bytes(params: Params, k_max: int) -> int:
+    out = ctypes.c_size_t(0)
+    rc = lib().lukv_importance_workspace_bytes(ctypes.byref(params), int(k_max), ctypes.byref(out))
+    if rc != OK:
+        raise LukvError(rc, "lukv_importance_workspace_bytes")
+    return int(out.value)
+
+
+def lukv_oracle_importance(params: Params, k_max: int, d_model: int, q_dec, k, v, k_dec, w_o, normalize: bool,
+                           importance, ws, stream=None, check: bool = True) -> int:
+    """Oracle importance (Sec. 4.1): q_dec [S][L][H*G][k_max][d], k, v [S][L][H][T][d], k_dec [S][L][H][k_max][d] or
+    None, w_o [L][H*G][d][d_model] -> importance [S][N][n] fp32 (all device)."""
+    rc = lib().lukv_oracle_importance(ctypes.byref(params), int(k_max), int(d_model), _ptr(q_dec), _ptr(k), _ptr(v),
+                                      _ptr(k_dec), _ptr(w_o), int(bool(normalize)), _ptr(importance), _ptr(ws),
+                                      0 if ws is None else ws.numel() * ws.element_size(), _stream(stream))
+    return _check(rc, "lukv_oracle_importance", check)
 
 
 def lukv_exact_workspace_bytes(params: Params, max_budget: int) -> int:

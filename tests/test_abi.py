@@ -128,6 +128,21 @@ def test_profile_argument_errors_come_back_before_any_launch():
     assert lukv.lukv_profile_budgets(p, None, grid, [0.5, 0.5], f, f, check=False) == lukv.ERR_INVALID_ARG
 
 
+def test_importance_argument_errors_come_back_before_any_launch():
+    p = _p()
+    f = _Fake()
+    assert lukv.lukv_importance_workspace_bytes(p, 8) > 0
+    assert lukv.lukv_importance_workspace_bytes(p, 64) > lukv.lukv_importance_workspace_bytes(p, 8)
+    with pytest.raises(lukv.LukvError):
+        lukv.lukv_importance_workspace_bytes(p, 0)
+    args = (f, f, f, None, f, True, f)
+    assert lukv.lukv_oracle_importance(p, 0, 16, *args, f, check=False) == lukv.ERR_INVALID_ARG
+    assert lukv.lukv_oracle_importance(p, 8, 0, *args, f, check=False) == lukv.ERR_INVALID_ARG
+    assert lukv.lukv_oracle_importance(p, 8, 16, None, f, f, None, f, True, f, f, check=False) == lukv.ERR_INVALID_ARG
+    assert lukv.lukv_oracle_importance(p, 8, 16, *args, _Fake(nbytes=16), check=False) == lukv.ERR_WORKSPACE_TOO_SMALL
+    assert lukv.lukv_oracle_importance(p, 8, 16, *args, _Fake(addr=0x10010), check=False) == lukv.ERR_INVALID_ARG
+
+
 def test_deployment_settings_are_validated():
     f = _Fake()
     p = _p(min_keep=0.5)                      # n = 248, floor 124 tokens per head, N = 4
