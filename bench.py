@@ -504,6 +504,23 @@ def run_profile_path(args):
     curves_ms = timed(lambda: lukv.lukv_build_curves(pc, c_scores, c_imp, c_out), max(args.steps // 2, 1), 3)
     del c_scores, c_imp, c_out
 
+    # oracle importance of one calibration query (decode queries, the cache, the output projection): 64 decode
+    # steps, model width 4096, every head of the workload's shape
+    Kd, Dm = 64, 4096
+    pi = lukv.make_params(1, wl.L, wl.H, wl.G, wl.d, Tc, wl.w, 1, wl.dtype, Tc + 1)
+    dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    i_q = torch.randn((1, wl.L, wl.H * wl.G, Kd, wl.d), generator=g, device="cuda").to(dt)
+    i_k = torch.randn((1, wl.L, wl.H, Tc, wl.d), generator=g, device="cuda").to(dt)
+    i_v = torch.randn((1, wl.L, wl.H, Tc, wl.d), generator=g, device="cuda").to(dt)
+    i_kd = torch.randn((1, wl.L, wl.H, Kd, wl.d), generator=g, device="cuda").to(dt)
+    i_wo = (torch.randn((wl.L, wl.H * wl.G, wl.d, Dm), generator=g, device="cuda") / wl.d ** 0.5).to(dt)
+    i_ws = torch.empty(lukv.lukv_importance_workspace_bytes(pi, Kd), dtype=torch.uint8, device="cuda")
+    i_out = torch.empty((1, wl.N, Tc - wl.w), dtype=torch.float32, device="cuda")
+    imp_ms = timed(lambda: lukv.lukv_oracle_importance(pi, Kd, Dm, i_q, i_k, i_v, i_kd, i_wo, True, i_out, i_ws), 3, 1)
+    imp_launches = lukv.lukv_last_launch_count()
+    imp_flops = 2.0 * wl.N * wl.G * (Tc - wl.w) * wl.d * Dm + 2.0 * 2 * wl.N * wl.G * Kd * Tc * wl.d
+    del i_q, i_k, i_v, i_kd, i_wo, i_ws, i_out
+
     build_ms = timed(lambda: lukv.lukv_profile_build(calib, U, Mq, ratios, phi, pws), args.steps, max(args.warmup, 3))
     build_launches = lukv.lukv_last_launch_count()
 
@@ -576,6 +593,9 @@ def run_profile_path(args):
         "exact_allocate": {"ms_per_call": exact_ms, "heads": wl.N, "positions": Tc - wl.w, "budget": Bx,
                            "launches": exact_launches, "optimum": exact_val, "greedy_on_raw_curves": greedy_raw,
                            "relaxation_gap": (exact_val - greedy_raw) / exact_val},
+        "oracle_importance": {"ms_per_call": imp_ms, "queries": 1, "heads": wl.N, "gqa_group": wl.G,
+                              "positions": Tc - wl.w, "decode_steps": Kd, "d_model": Dm, "launches": imp_launches,
+                              "flops": imp_flops, "tflops": imp_flops / (imp_ms * 1e-3) / 1e12},
         "build_curves": {"ms_per_call": curves_ms, "queries": Mq, "heads": wl.N, "positions": Tc - wl.w,
                          "compares": float(Mq) * wl.N * (Tc - wl.w) ** 2},
         "online_mode": {"metric": METRIC, "value": wl.S * wl.T / (online_ms * 1e-3), "unit": UNIT,

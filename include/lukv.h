@@ -178,6 +178,28 @@ LUKV_API int lukv_compress(const lukv_params_t* params, const void* q_win, const
                   size_t ws_bytes, void* stream);
 
 /*
+ * The same for a batch whose sequences have different context lengths, in one set of launches (App. E runs the
+ * method on whatever context a request brings; Sec. 5.3: budgets are known before prefill, so nothing forces
+ * sequences of one length into a call).  Sequence q has ctx_lens[q] cached positions, w < ctx_lens[q] <= T, of
+ * which the last w are its observation window and the first n_q = ctx_lens[q] - w are rankable.
+ *   - params->ctx_len = T is the ROW STRIDE of the cache: k, v are [S][L][H][T][d] with sequence q using the
+ *     first ctx_lens[q] rows of each of its heads (the rest is padding and is never read as data);
+ *     scores (lukv_score_ragged) are [S][N][T-w] with the first n_q entries of a row written.
+ *   - The curve grid is per sequence: segment size ctx_lens[q]/(P-1), so (P-1) must divide every length
+ *     (LUKV_ERR_UNSUPPORTED otherwise); 0 <= B_q <= N*n_q; min_keep gives ceil(min_keep*n_q) per head of q.
+ *   - Outputs as in lukv_compress: head u of sequence q keeps budgets[u] positions of [0, n_q) and its window rows
+ *     n_q .. ctx_lens[q]-1; rows = sum_q B_q + S*N*w.
+ * ctx_lens [S] int32, HOST, read before the call returns; S <= 64.  The result equals what S single-sequence
+ * calls (params with batch 1 and ctx_len = ctx_lens[q]) would produce, concatenated.
+ */
+LUKV_API int lukv_score_ragged(const lukv_params_t* params, const int32_t* ctx_lens, const void* q_win, const void* k,
+                               float* scores, void* ws, size_t ws_bytes, void* stream);
+LUKV_API int lukv_compress_ragged(const lukv_params_t* params, const int32_t* ctx_lens, const void* q_win,
+                                  const void* k, const void* v, const float* curves, const int64_t* budgets_in,
+                                  void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets, int32_t* offsets,
+                                  int64_t rows_cap, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Profiling variant of lukv_compress (the paper has no counterpart): same arguments and
  * results, but a CUDA event is recorded after every kernel and the call SYNCHRONISES the
  * stream before returning the per-kernel device times.  Not for production use.

@@ -187,6 +187,30 @@ def compress(q, k, v, curves, budgets_in, G: int, kp: int, scale: float = 0.0, n
     return out
 
 
+def compress_ragged(q, k, v, curves, budgets_in, ctx_lens, G: int, kp: int, scale: float = 0.0, n_sink: int = 0,
+                    min_keep: float = 0.0):
+    """A batch whose sequences have different context lengths (App. E applies the method to whatever context a
+    request brings): k, v [S][L][H][T_max][d] with sequence s using the first ctx_lens[s] positions, its window
+    being the last w of those.  By definition the result of one single-sequence call per sequence, concatenated:
+    budgets [S][N], offsets [S*N+1] (running over all sequences), kept_idx / k_out / v_out in sequence order,
+    scores as a list of [N][ctx_lens[s]-w] arrays."""
+    q, k, v = _c(q), _c(k), _c(v)
+    budgets_in = _c(budgets_in, np.int64)
+    S = q.shape[0]
+    parts = [compress(q[s:s + 1], np.ascontiguousarray(k[s:s + 1, :, :, :int(ctx_lens[s])]),
+                      np.ascontiguousarray(v[s:s + 1, :, :, :int(ctx_lens[s])]), curves, budgets_in[s:s + 1], G, kp,
+                      scale=scale, n_sink=n_sink, min_keep=min_keep) for s in range(S)]
+    offsets, base = [np.zeros(1, np.int32)], 0
+    for part in parts:
+        offsets.append((part["offsets"][1:].astype(np.int64) + base).astype(np.int32))
+        base += int(part["offsets"][-1])
+    return dict(k_out=np.concatenate([part["k_out"] for part in parts]),
+                v_out=np.concatenate([part["v_out"] for part in parts]),
+                kept_idx=np.concatenate([part["kept_idx"] for part in parts]),
+                budgets=np.concatenate([part["budgets"] for part in parts]),
+                offsets=np.concatenate(offsets), scores=[part["scores"][0] for part in parts])
+
+
 def profile_build(curves, T: int, w: int, ratios, min_keep: float = 0.0):
     """Offline profile (Sec. 4.3, Eq. "calibration_avg"). curves [Mq][N][P] -> profile [R][N] fp32."""
     curves = _c(curves, np.float32)

@@ -104,6 +104,8 @@ constexpr int kSeqPerLaunch = 32;
 struct GreedyArgs {
   long long budget[kSeqPerLaunch];    // B_q
   long long row_base[kSeqPerLaunch];  // packed rows before sequence q
+  int T[kSeqPerLaunch];               // context length of sequence q (the curve grid is T/(P-1) tokens per segment)
+  int floor_tok[kSeqPerLaunch];       // tokens every head of sequence q keeps at least
   int seq0;                           // first sequence of this launch
 };
 
@@ -153,8 +155,10 @@ __device__ __forceinline__ long long block_sum_ll(long long v, long long* buf) {
 __global__ void __launch_bounds__(kGreedyMaxThreads) greedy_kernel(const float* __restrict__ gains, GreedyArgs args,
                                                                    int32_t* __restrict__ budgets,
                                                                    int32_t* __restrict__ offsets, SetStride set,
-                                                                   int N, int P, int seg, int nseg, int n, int w,
-                                                                   int floor_tok) {
+                                                                   int N, int P, int w) {
+  // the sequence's own grid: n rankable positions, seg tokens per curve segment, nseg segments with capacity
+  const int n = args.T[blockIdx.x] - w, seg = args.T[blockIdx.x] / (P - 1), nseg = (n + seg - 1) / seg;
+  const int floor_tok = args.floor_tok[blockIdx.x];
   gains += (size_t)blockIdx.y * set.gains;
   budgets += (size_t)blockIdx.y * set.budgets;
   offsets += (size_t)blockIdx.y * set.offsets;
@@ -283,15 +287,21 @@ cudaError_t launch_greedy(const Dims& dm, const float* gains, const int64_t* bud
     for (int i = 0; i < kSeqPerLaunch; ++i) {
       args.budget[i] = 0;
       args.row_base[i] = 0;
+      args.T[i] = dm.T;
+      args.floor_tok[i] = dm.floor_tok;
     }
     for (int i = 0; i < cnt; ++i) {
       args.budget[i] = budgets_host[q0 + i];
       args.row_base[i] = base;
+      if (dm.seq_T) {
+        args.T[i] = dm.seq_T[q0 + i];
+        args.floor_tok[i] = seq_floor_tokens(dm, q0 + i);
+      }
       base += budgets_host[q0 + i] + (long long)dm.N * dm.w;
     }
     args.seq0 = q0;
     greedy_kernel<<<dim3(cnt, n_sets), threads, greedy_smem, lc.st>>>(gains, args, budgets, offsets, set, dm.N, dm.P,
-                                                                      dm.seg, dm.nseg, dm.n, dm.w, dm.floor_tok);
+                                                                      dm.w);
     lc.mark("greedy");
   }
   return cudaGetLastError();

@@ -39,6 +39,20 @@ Workspace carve_workspace(const Dims& dm, void* base) {
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Per-sequence context lengths of a ragged call: w < T_q <= T, the curve grid must divide every length, the sinks
+// must fit every sequence.  On success dm describes the longest sequence and carries the lengths.
+static int attach_seq_lens(Dims* dm, const int32_t* ctx_lens) {
+  if (!ctx_lens) return LUKV_ERR_INVALID_ARG;
+  if (dm->S > kMaxRaggedSeqs) return LUKV_ERR_UNSUPPORTED;
+  for (int q = 0; q < dm->S; ++q) {
+    const int Tq = ctx_lens[q];
+    if (Tq <= dm->w || Tq > dm->T || dm->n_sink > Tq - dm->w) return LUKV_ERR_INVALID_ARG;
+    if (Tq % (dm->P - 1) != 0) return LUKV_ERR_UNSUPPORTED;
+  }
+  dm->seq_T = ctx_lens;
+  return LUKV_OK;
+}
+
 // Validates the parameter block and fills Dims.
 static int make_dims(const lukv_params_t* p, Dims* dm) {
   if (!p) return LUKV_ERR_INVALID_ARG;
@@ -72,6 +86,8 @@ static int make_dims(const lukv_params_t* p, Dims* dm) {
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : (float)(1.0 / sqrt((double)dm->d));
   dm->scale_log2 = (float)((double)scale * 1.4426950408889634);
   dm->n_sink = p->n_sink;
+  dm->min_keep = p->min_keep;
+  dm->seq_T = nullptr;
   const double fl = ceil((double)p->min_keep * (double)dm->n);
   dm->floor_tok = fl < 0.0 ? 0 : (fl > (double)dm->n ? dm->n : (int)fl);
   return LUKV_OK;
@@ -80,7 +96,8 @@ static int make_dims(const lukv_params_t* p, Dims* dm) {
 static int check_budgets(const Dims& dm, const int64_t* budgets_in, int64_t* total_rows) {
   int64_t rows = 0;
   for (int q = 0; q < dm.S; ++q) {
-    if (budgets_in[q] < (int64_t)dm.N * dm.floor_tok || budgets_in[q] > (int64_t)dm.N * dm.n) return LUKV_ERR_BUDGET;
+    if (budgets_in[q] < (int64_t)dm.N * seq_floor_tokens(dm, q) || budgets_in[q] > (int64_t)dm.N * seq_rankable(dm, q))
+      return LUKV_ERR_BUDGET;
     rows += budgets_in[q] + (int64_t)dm.N * dm.w;
   }
   *total_rows = rows;
@@ -182,9 +199,11 @@ static int run_compress(const Dims& dm, const void* q_win, const void* k, const 
 static int check_compress_args(const lukv_params_t* params, const void* q_win, const void* k, const void* v,
                                const float* curves, const int64_t* budgets_in, void* k_out, void* v_out,
                                int32_t* kept_idx, int32_t* budgets, int32_t* offsets, int64_t rows_cap, void* ws,
-                               size_t ws_bytes, Dims* dm, Workspace* w) {
+                               size_t ws_bytes, Dims* dm, Workspace* w, const int32_t* ctx_lens = nullptr,
+                               bool ragged = false) {
   int rc = make_dims(params, dm);
   if (rc != LUKV_OK) return rc;
+  if (ragged && (rc = attach_seq_lens(dm, ctx_lens)) != LUKV_OK) return rc;
   if (!q_win || !k || !v || !curves || !budgets_in || !k_out || !v_out || !kept_idx || !budgets || !offsets ||
       !aligned16(q_win) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
     return LUKV_ERR_INVALID_ARG;
@@ -215,6 +234,22 @@ int lukv_score(const lukv_params_t* params, const void* q_win, const void* k, fl
   Dims dm;
   int rc = make_dims(params, &dm);
   if (rc != LUKV_OK) return rc;
+  if (!q_win || !k || !scores || !aligned16(q_win) || !aligned16(k)) return LUKV_ERR_INVALID_ARG;
+  Workspace w;
+  if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  if (run_score(dm, q_win, k, w, scores, nullptr, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
+}
+
+int lukv_score_ragged(const lukv_params_t* params, const int32_t* ctx_lens, const void* q_win, const void* k,
+                      float* scores, void* ws, size_t ws_bytes, void* stream) {
+  Dims dm;
+  int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if ((rc = attach_seq_lens(&dm, ctx_lens)) != LUKV_OK) return rc;
   if (!q_win || !k || !scores || !aligned16(q_win) || !aligned16(k)) return LUKV_ERR_INVALID_ARG;
   Workspace w;
   if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
@@ -271,6 +306,23 @@ int lukv_compress(const lukv_params_t* params, const void* q_win, const void* k,
   Workspace w;
   int rc = check_compress_args(params, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets,
                                rows_cap, ws, ws_bytes, &dm, &w);
+  if (rc != LUKV_OK) return rc;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  rc = run_compress(dm, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets, rows_cap,
+                    dev_status, w, lc, true);
+  if (rc == LUKV_OK) g_last_launches = lc.launches;
+  return rc;
+}
+
+int lukv_compress_ragged(const lukv_params_t* params, const int32_t* ctx_lens, const void* q_win, const void* k,
+                         const void* v, const float* curves, const int64_t* budgets_in, void* k_out, void* v_out,
+                         int32_t* kept_idx, int32_t* budgets, int32_t* offsets, int64_t rows_cap, int32_t* dev_status,
+                         void* ws, size_t ws_bytes, void* stream) {
+  Dims dm;
+  Workspace w;
+  int rc = check_compress_args(params, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets,
+                               rows_cap, ws, ws_bytes, &dm, &w, ctx_lens, true);
   if (rc != LUKV_OK) return rc;
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;

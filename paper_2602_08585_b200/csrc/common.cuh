@@ -3,6 +3,7 @@
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <math.h>
 #include <stddef.h>
 #include <stdint.h>
 
@@ -21,6 +22,10 @@ struct Dims {
   float scale_log2;  // softmax scale * log2(e): logits are kept in the exp2 domain
   int n_sink;        // leading positions that rank first in the selection
   int floor_tok;     // tokens every head keeps at least: ceil(min_keep * n)
+  // Sequences of different lengths in one call: seq_T[q] (HOST, S entries) is the context length of sequence q;
+  // T, n and the tensor strides then describe the longest one.  nullptr: every sequence has length T.
+  const int32_t* seq_T = nullptr;
+  float min_keep = 0.f;  // as given (the per-sequence floors of a ragged call are derived from it)
   int64_t heads() const { return (int64_t)S * N; }
   size_t esize() const { return dtype == LUKV_DTYPE_BF16 ? 2 : 4; }
 };
@@ -51,6 +56,23 @@ Workspace carve_workspace(const Dims& dm, void* base);  // base may be null (siz
 // Heads per sequence the greedy kernel can hold: 12 bytes of shared memory each, 227 KB per CTA
 // less its static arrays.
 constexpr int kGreedyMaxHeads = 18944;
+
+// Most sequences a call with per-sequence context lengths takes: their lengths travel by value in the launch
+// arguments of the kernels.
+constexpr int kMaxRaggedSeqs = 64;
+struct SeqLens {
+  int T[kMaxRaggedSeqs];
+};
+
+// Rankable positions and minimum retention (tokens) of sequence q: the call's own when all sequences have one
+// length, else from its length (the floor is ceil(min_keep * n) in fp64, as in the uniform case).
+inline int seq_rankable(const Dims& dm, int q) { return dm.seq_T ? dm.seq_T[q] - dm.w : dm.n; }
+inline int seq_floor_tokens(const Dims& dm, int q) {
+  if (!dm.seq_T) return dm.floor_tok;
+  const int n = dm.seq_T[q] - dm.w;
+  const double fl = ceil((double)dm.min_keep * (double)n);
+  return fl < 0.0 ? 0 : (fl > (double)n ? n : (int)fl);
+}
 
 // Launch bookkeeping: counts the kernels a call enqueues and, when a timeline is attached
 // (profiling entry point only), records a CUDA event after each of them.

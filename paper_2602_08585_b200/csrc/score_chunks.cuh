@@ -52,7 +52,8 @@ __device__ __forceinline__ void p1_chunk(const float (&v)[32], int jbase, int li
   m = mn;
 }
 
-// Pass 2, 32 columns (query rows c0..c0+31) of one key: add the probabilities.
+// Pass 2, 32 columns (query rows c0..c0+31) of one key: add the probabilities.  The -lse of the rows is read from
+// shared memory.
 __device__ __forceinline__ void p2_chunk(const float (&v)[32], const float* nlse, uint64_t sc2, uint64_t& acc0,
                                          uint64_t& acc1) {
 #pragma unroll
@@ -61,6 +62,24 @@ __device__ __forceinline__ void p2_chunk(const float (&v)[32], const float* nlse
     acc0 = fadd2(acc0, ex2_pair(ffma2(pack2(v[i], v[i + 1]), sc2, ls.x)));
     if (LUKV_POLY_SEL2(i)) acc1 = fadd2(acc1, ex2_poly_pair<false>(ffma2(pack2(v[i + 2], v[i + 3]), sc2, ls.y)));
     else acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(v[i + 2], v[i + 3]), sc2, ls.y)));
+  }
+}
+
+// Variant for the micro-benchmark's comparison: the -lse values come out of registers (lane l of the warp holds
+// rows 4l..4l+3 of a block of 128 rows in `mine`; every lane fetches the four it needs next by shuffles; c0 is a
+// multiple of 32 below 128).  With the tensor pipe streaming operands out of shared memory all the time this is
+// much faster in isolation (1111 against 1810 clocks per tile), but inside the scorer, where the pipe is busy
+// under half of the time and the shuffles cost issue slots, it was slower (0.827 against 0.797 ms).
+__device__ __forceinline__ void p2_chunk_shfl(const float (&v)[32], const float4 mine, int c0, uint64_t sc2, uint64_t& acc0,
+                                              uint64_t& acc1) {
+#pragma unroll
+  for (int i = 0; i < 32; i += 4) {
+    const int src = (c0 + i) >> 2;
+    const float l0 = __shfl_sync(0xffffffffu, mine.x, src), l1 = __shfl_sync(0xffffffffu, mine.y, src);
+    const float l2 = __shfl_sync(0xffffffffu, mine.z, src), l3 = __shfl_sync(0xffffffffu, mine.w, src);
+    acc0 = fadd2(acc0, ex2_pair(ffma2(pack2(v[i], v[i + 1]), sc2, pack2(l0, l1))));
+    if (LUKV_POLY_SEL2(i)) acc1 = fadd2(acc1, ex2_poly_pair<false>(ffma2(pack2(v[i + 2], v[i + 3]), sc2, pack2(l2, l3))));
+    else acc1 = fadd2(acc1, ex2_pair(ffma2(pack2(v[i + 2], v[i + 3]), sc2, pack2(l2, l3))));
   }
 }
 

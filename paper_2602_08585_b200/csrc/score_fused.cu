@@ -95,6 +95,12 @@ struct FusedArgs {
   int lag;             // 2..kMaxLag: pass 1 of item k+lag-1 precedes pass 2 of item k
   int l2_hints;        // 1: pass-1 key loads ask L2 to keep the lines, pass-2 loads to drop them first
   float scale_log2;
+  // sequences of different lengths in one launch (RAGGED kernels): seq_T[q] = context length of sequence q,
+  // seq_item0[q] = number of its first work item; heads_per_seq heads each.  The uniform fields above then hold
+  // the maxima (strides and capacities).  The tables travel by value in the launch arguments.
+  int seq_T[kMaxRaggedSeqs], seq_item0[kMaxRaggedSeqs];
+  int n_seq, heads_per_seq, total_items;
+  int T_stride, n_stride;  // rows between consecutive heads in K and in the raw scores
   uint32_t spin_limit; // iterations a wait may take
   int drop_item;       // test hook: this work item's partials are stored but never counted in (-1: none)
 };
@@ -104,33 +110,56 @@ struct Job {
   int c;       // item of the head
   int tile0;   // first key tile
   int ntiles;  // key tiles of this job (may be 0)
+  int n;       // rankable positions of the head
+  int iph;     // work items of the head
   bool p2;
 };
 
+template <bool RAGGED>
 __device__ __forceinline__ Job make_job(int k, bool p2, const FusedArgs& a) {
   Job j;
   j.p2 = p2;
   const int item = (int)blockIdx.x + k * (int)gridDim.x;
-  const int hu = item / a.items_per_head;
-  j.c = item - hu * a.items_per_head;
-  j.u = a.head0 + hu;
+  int tiles_T = a.tiles_T, tiles_n = a.tiles_n;
+  if (!RAGGED) {
+    j.n = a.n;
+    j.iph = a.items_per_head;
+    const int hu = item / a.items_per_head;
+    j.c = item - hu * a.items_per_head;
+    j.u = a.head0 + hu;
+  } else {
+    int lo = 0, hi = a.n_seq;  // the sequence whose items contain `item`
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (a.seq_item0[mid] <= item) lo = mid; else hi = mid;
+    }
+    const int2 sq = make_int2(a.seq_T[lo], a.seq_item0[lo]);
+    j.n = sq.x - a.w;
+    tiles_T = (sq.x + kTileKeys - 1) / kTileKeys;
+    tiles_n = (j.n + kTileKeys - 1) / kTileKeys;
+    j.iph = (tiles_T + a.item_tiles - 1) / a.item_tiles;
+    const int local = item - sq.y, hu = local / j.iph;
+    j.c = local - hu * j.iph;
+    j.u = lo * a.heads_per_seq + hu;
+  }
   j.tile0 = j.c * a.item_tiles;
-  const int lim = p2 ? a.tiles_n : a.tiles_T;
+  const int lim = p2 ? tiles_n : tiles_T;
   j.ntiles = max(0, min(a.item_tiles, lim - j.tile0));
   return j;
 }
 
 // Job `idx` of a CTA that owns K items: lag-1 pass-1 jobs first, then pass 1 of item k+lag-1
 // alternating with pass 2 of item k, then the remaining pass-2 jobs.
+template <bool RAGGED>
 __device__ __forceinline__ Job decode_job(int idx, int K, const FusedArgs& a) {
   const int lead = min(a.lag - 1, K);
-  if (idx < lead) return make_job(idx, false, a);
+  if (idx < lead) return make_job<RAGGED>(idx, false, a);
   const int r = idx - lead, pairs = 2 * (K - lead);
-  if (r < pairs) return (r & 1) ? make_job(r >> 1, true, a) : make_job(lead + (r >> 1), false, a);
-  return make_job(K - lead + (r - pairs), true, a);
+  if (r < pairs) return (r & 1) ? make_job<RAGGED>(r >> 1, true, a) : make_job<RAGGED>(lead + (r >> 1), false, a);
+  return make_job<RAGGED>(K - lead + (r - pairs), true, a);
 }
 
-template <int MT, int NQ>
+template <int MT, int NQ, bool RAGGED>
 __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
     score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                        const FusedArgs a) {
@@ -152,7 +181,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
   float* nlse_s = reinterpret_cast<float*>(smem + P::kLseOff);    // [kMaxLag][256]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_items = a.nheads * a.items_per_head;
+  const int total_items = a.total_items;
   const int K = (total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // items of this CTA (>= 1)
   const int njobs = 2 * K;
 
@@ -194,7 +223,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
       const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
       uint32_t tt = 0, jq = 0;
       for (int idx = 0; idx < njobs; ++idx) {
-        const Job j = decode_job(idx, K, a);
+        const Job j = decode_job<RAGGED>(idx, K, a);
         if (j.ntiles == 0) continue;
         const uint32_t slot = jq % P::kQSlots;
         if (!mbar_wait(bar(P::kBarQEmpty, slot), ((jq / P::kQSlots) & 1) ^ 1, abort_flag, a.dev_status, a.spin_limit)) break;
@@ -212,7 +241,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
           const uint32_t s = tt % kStages, ph = (tt / kStages) & 1;
           if (!(ok = mbar_wait(bar(P::kBarEmpty, s), ph ^ 1, abort_flag, a.dev_status, a.spin_limit))) break;
           mbar_expect_tx(bar(P::kBarFull, s), kStageBytes);
-          const int row = j.u * a.T + (j.tile0 + t) * kTileKeys;
+          const int row = j.u * a.T_stride + (j.tile0 + t) * kTileKeys;
           const uint32_t dst = k_s + s * kStageBytes;
           if (a.l2_hints) {
             const uint64_t pol = j.p2 ? drop : keep;
@@ -236,7 +265,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
       const uint32_t me = warp == kEpiWarps + 1 ? 0u : 1u;
       uint32_t tt = 0, jq = 0;
       for (int idx = 0; idx < njobs; ++idx) {
-        const Job j = decode_job(idx, K, a);
+        const Job j = decode_job<RAGGED>(idx, K, a);
         if (j.ntiles == 0) continue;
         const uint32_t slot = jq % P::kQSlots;
         const uint32_t qd = q_s + slot * P::kQBytes;
@@ -309,7 +338,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
         if (ready) {
           const int k = kp;
           const bool ok = true;
-          const Job j1 = make_job(k, false, a);
+          const Job j1 = make_job<RAGGED>(k, false, a);
           if (ok) {
             // one value per row: the log-sum-exp of the item's keys, m + log2(l); -inf for an empty partial
             float* dst = a.stats + ((size_t)j1.u * a.items_per_head + j1.c) * kRowsPad;
@@ -338,7 +367,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
           int last = 0;
           const bool dropped = (int)blockIdx.x + k * (int)gridDim.x == a.drop_item;
           if (lane == 0 && ok && !dropped && !*abort_flag)
-            last = atom_add_acq_rel(a.head_cnt + j1.u, 1) == a.items_per_head - 1;
+            last = atom_add_acq_rel(a.head_cnt + j1.u, 1) == j1.iph - 1;
           last = __shfl_sync(0xffffffffu, last, 0);
           if (last) {
             // Fold the head's partials into lse = log2(sum_c 2^(v_c)).  The bulk-copy engine brings them
@@ -349,9 +378,9 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
             // the fallback when that sum leaves a safe range.
             constexpr int kVecs = MT;  // float4 per lane and item
             const char* src = reinterpret_cast<const char*>(a.stats) + (size_t)j1.u * a.items_per_head * kRowsPad * 4;
-            const int nblk = (a.items_per_head + P::kFinParts - 1) / P::kFinParts;
+            const int nblk = (j1.iph + P::kFinParts - 1) / P::kFinParts;
             auto request = [&](int blk) {  // lane 0
-              const int parts = min(P::kFinParts, a.items_per_head - blk * P::kFinParts);
+              const int parts = min(P::kFinParts, j1.iph - blk * P::kFinParts);
               const uint32_t bytes = (uint32_t)parts * kRowsPad * 4;
               mbar_expect_tx(bar(P::kBarFin, 0), bytes);
               bulk_load(sbase + P::kFinOff, src + (size_t)blk * P::kFinParts * kRowsPad * 4, bytes, bar(P::kBarFin, 0));
@@ -367,7 +396,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
                 fin_ok = mbar_wait(bar(P::kBarFin, 0), fin_uses[0] & 1, abort_flag, a.dev_status, a.spin_limit);
                 ++fin_uses[0];
                 if (!fin_ok) break;
-                const int parts = min(P::kFinParts, a.items_per_head - blk * P::kFinParts);
+                const int parts = min(P::kFinParts, j1.iph - blk * P::kFinParts);
                 if (blk == 0) {
 #pragma unroll
                   for (int vv = 0; vv < kVecs; ++vv) {
@@ -380,7 +409,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
                   // the fallback needs the maximum of every row first; it is rare, so it simply reads the
                   // partials from global memory
                   const float4* g = reinterpret_cast<const float4*>(src);
-                  for (int c = 0; c < a.items_per_head; ++c)
+                  for (int c = 0; c < j1.iph; ++c)
 #pragma unroll
                     for (int vv = 0; vv < kVecs; ++vv) {
                       const float4 v = __ldcg(g + (size_t)c * (kRowsPad / 4) + vv * 32 + lane);
@@ -427,7 +456,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
         }
       }
       if (kf < kp) {
-        const Job j2 = make_job(kf, true, a);
+        const Job j2 = make_job<RAGGED>(kf, true, a);
         if (j2.ntiles == 0) {
           ++kf;
           progress = true;
@@ -481,12 +510,12 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
     const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2);
     uint32_t tt = 0, p1c = 0, p2c = 0;
     for (int idx = 0; idx < njobs; ++idx) {
-      const Job j = decode_job(idx, K, a);
+      const Job j = decode_job<RAGGED>(idx, K, a);
       if (j.ntiles == 0) continue;
       if (!j.p2) {
         // ---- pass 1: (reference, sum-exp) of this thread's query row over the job's keys
         const int r = (MT == 2 ? 128 * quad : 0) + qtid;
-        const int lim = r < a.M ? a.n + (r % a.w) : -1;           // last visible key; -1: padded row
+        const int lim = r < a.M ? j.n + (r % a.w) : -1;           // last visible key; -1: padded row
         float m = -INFINITY, l = 0.f;
         for (int t = 0; t < j.ntiles; ++t, ++tt) {
           if (MT == 1 && (int)(tt % NQ) != quad) continue;
@@ -495,7 +524,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
           if (ok) {
             tc_fence_after();
             const int j0 = (j.tile0 + t) * kTileKeys;
-            const bool masked = j0 + kTileKeys > a.n;             // tile reaches into the window / past T
+            const bool masked = j0 + kTileKeys > j.n;             // tile reaches into the window / past T
             const uint32_t tcol = tmem_base + lane_addr + buf * P::kBufCols + (MT == 2 ? 128 * quad : 0);
             float va[32], vb[32];
             tmem_ld32(tcol, va);
@@ -556,7 +585,7 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(P::kBarTEmpty, buf), MT == 2 ? 2 : 1);
-            if (key < a.n) a.raw[(size_t)j.u * a.n + key] = sum4(acc0, acc1);
+            if (key < j.n) a.raw[(size_t)j.u * a.n_stride + key] = sum4(acc0, acc1);
           }
         }
         __syncwarp();
@@ -581,11 +610,12 @@ __global__ void __launch_bounds__(Plan<MT, NQ>::kThreads, 1)
 
 // ---- host side --------------------------------------------------------------------------------
 
-template <int MT, int NQ>
-cudaError_t launch_fused(const CUtensorMap& qm, const CUtensorMap& km, FusedArgs args, int spare_sms, LaunchCtx& lc) {
+template <int MT, int NQ, bool RAGGED = false>
+cudaError_t launch_fused(const CUtensorMap& qm, const CUtensorMap& km, FusedArgs args, int spare_sms, LaunchCtx& lc,
+                         const int32_t* seq_T_host = nullptr) {
   using P = Plan<MT, NQ>;
   const int smem = P::kTotal;
-  auto kern = score_fused_kernel<MT, NQ>;
+  auto kern = score_fused_kernel<MT, NQ, RAGGED>;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
   int dev = 0, sms = 0, per_sm = 0;
@@ -619,7 +649,18 @@ cudaError_t launch_fused(const CUtensorMap& qm, const CUtensorMap& km, FusedArgs
   }
   while ((args.tiles_T + args.item_tiles - 1) / args.item_tiles > sms) ++args.item_tiles;
   args.items_per_head = (args.tiles_T + args.item_tiles - 1) / args.item_tiles;
-  const int total_items = args.nheads * args.items_per_head;
+  int total_items = args.nheads * args.items_per_head;
+  if (RAGGED) {
+    int base = 0;
+    for (int q = 0; q < args.n_seq; ++q) {
+      args.seq_T[q] = seq_T_host[q];
+      args.seq_item0[q] = base;
+      const int tiles = (seq_T_host[q] + kTileKeys - 1) / kTileKeys;
+      base += args.heads_per_seq * ((tiles + args.item_tiles - 1) / args.item_tiles);
+    }
+    total_items = base;
+  }
+  args.total_items = total_items;
   const int grid = total_items < sms ? total_items : sms;  // one CTA per SM: each owns the SM's tensor memory
   void* params[] = {(void*)&qm, (void*)&km, (void*)&args};
   // cooperative launch: the CTAs of a head wait for one another, so all must be resident
@@ -673,7 +714,7 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
   // shape allows it (it parks a head's exponentials in tensor memory and is bound by the latency of the
   // log-sum-exp exchange between CTAs; at long contexts the two sweeps are faster).
   const char* which = getenv("LUKV_SCORER");
-  if (which && which[0] == 'o' && score_onepass_eligible(dm)) {
+  if (which && which[0] == 'o' && !dm.seq_T && score_onepass_eligible(dm)) {
     const cudaError_t e1 = launch_score_onepass(dm, q, k, ws, dev_status, hr, clear_flags, spare_sms, lc);
     if (e1 != cudaErrorNotSupported) return e1;
   }
@@ -690,6 +731,10 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
   args.T = dm.T;
   args.w = dm.w;
   args.n = dm.n;
+  args.T_stride = dm.T;
+  args.n_stride = dm.n;
+  args.n_seq = dm.S;
+  args.heads_per_seq = dm.N;
   args.lse_rows = (dm.M + 3) & ~3;
   args.head0 = hr.h0;
   args.nheads = hr.nh;
@@ -709,6 +754,12 @@ cudaError_t launch_score_tc(const Dims& dm, const void* q, const void* k, const 
   if (clear_flags) {
     const cudaError_t e = cudaMemsetAsync(ws.head_flags, 0, score_tc_flag_bytes(dm), lc.st);
     if (e != cudaSuccess) return e;
+  }
+  if (dm.seq_T) {
+    // sequences of different lengths: the whole call in one launch (no head ranges), work items dealt per sequence
+    if (hr.h0 != 0 || hr.nh != (int)dm.heads() || dm.S > kMaxRaggedSeqs) return cudaErrorInvalidValue;
+    return dm.M > 128 ? launch_fused<2, 2, true>(qm, km, args, spare_sms, lc, dm.seq_T)
+                      : launch_fused<1, 2, true>(qm, km, args, spare_sms, lc, dm.seq_T);
   }
   if (dm.M > 128) return launch_fused<2, 2>(qm, km, args, spare_sms, lc);
   static const int quads = env_int("LUKV_QUADS", 2, 3, 2);

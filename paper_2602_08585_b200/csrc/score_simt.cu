@@ -23,7 +23,7 @@ template <typename TIn, int D, int RPT, bool SWEEP2>
 __global__ void __launch_bounds__(kThreads) score_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k,
                                                               float* __restrict__ stats, const float* __restrict__ lse,
                                                               float* __restrict__ raw, int M, int T, int w, int chunks,
-                                                              float scale_log2) {
+                                                              float scale_log2, SeqLens sl, int heads_per_seq) {
   constexpr int kPitch = D + 4;
   extern __shared__ __align__(16) float smem[];
   float* Qs = smem;                         // [16*RPT][kPitch]
@@ -31,7 +31,9 @@ __global__ void __launch_bounds__(kThreads) score_simt_kernel(const TIn* __restr
   __shared__ float colred[kThreads / 32][kKeyTile];
 
   const int u = blockIdx.x / chunks, chunk = blockIdx.x % chunks;
-  const int n = T - w;
+  // T is the row stride of the cache (the longest sequence); Tu the length of this head's sequence
+  const int Tu = heads_per_seq > 0 ? sl.T[u / heads_per_seq] : T;
+  const int n = Tu - w, n_stride = T - w;
   const int tid = threadIdx.x, kg = tid & 15, rg = tid >> 4;
   const TIn* qh = q + (size_t)u * M * D;
   const TIn* kh = k + (size_t)u * T * D;
@@ -51,10 +53,10 @@ __global__ void __launch_bounds__(kThreads) score_simt_kernel(const TIn* __restr
   }
 
   const int key_begin = chunk * kChunk;
-  const int key_end = min(T, key_begin + kChunk);
+  const int key_end = min(Tu, key_begin + kChunk);
   for (int j0 = key_begin; j0 < key_end; j0 += kKeyTile) {
     __syncthreads();  // previous tile fully consumed (and Qs visible on the first pass)
-    load_rows_f32<TIn, D>(Ks, kh + (size_t)j0 * D, kKeyTile, min(kKeyTile, T - j0));
+    load_rows_f32<TIn, D>(Ks, kh + (size_t)j0 * D, kKeyTile, min(kKeyTile, Tu - j0));
     __syncthreads();
 
     float acc[RPT][4];
@@ -121,7 +123,7 @@ __global__ void __launch_bounds__(kThreads) score_simt_kernel(const TIn* __restr
 #pragma unroll
         for (int wv = 0; wv < kThreads / 32; ++wv) s += colred[wv][tid];
         const int j = j0 + tid;
-        if (j < n) raw[(size_t)u * n + j] = s;
+        if (j < n) raw[(size_t)u * n_stride + j] = s;
       }
     }
   }
@@ -169,16 +171,19 @@ __global__ void score_lse_kernel(const float* __restrict__ stats, float* __restr
   }
 }
 
-__global__ void max_pool_kernel(const float* __restrict__ raw, float* __restrict__ pooled, int n, int half,
-                                int tiles, int head0) {
+// n: row stride of the score arrays (the longest sequence); the head's own length comes from `sl` when the
+// sequences differ (heads_per_seq > 0).
+__global__ void max_pool_kernel(const float* __restrict__ raw, float* __restrict__ pooled, int n_stride, int half,
+                                int tiles, int head0, SeqLens sl, int heads_per_seq, int w) {
   const int u = head0 + blockIdx.x / tiles;
   const int j = (blockIdx.x % tiles) * blockDim.x + threadIdx.x;
+  const int n = heads_per_seq > 0 ? sl.T[u / heads_per_seq] - w : n_stride;
   if (j >= n) return;
-  const float* r = raw + (size_t)u * n;
+  const float* r = raw + (size_t)u * n_stride;
   const int lo = max(0, j - half), hi = min(n - 1, j + half);
   float best = r[lo];
   for (int t = lo + 1; t <= hi; ++t) best = fmaxf(best, r[t]);
-  pooled[(size_t)u * n + j] = best;
+  pooled[(size_t)u * n_stride + j] = best;
 }
 
 // The same pooling, four outputs per thread with 16-byte accesses, for rows whose length is a multiple
@@ -219,13 +224,17 @@ cudaError_t launch_sweeps(const Dims& dm, const void* q, const void* k, const Wo
   if ((e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   const unsigned grid = (unsigned)(dm.heads() * chunks);
+  SeqLens sl = {};
+  const int heads_per_seq = dm.seq_T ? dm.N : 0;
+  if (dm.seq_T)
+    for (int q = 0; q < dm.S; ++q) sl.T[q] = dm.seq_T[q];
   k1<<<grid, kThreads, smem, st>>>((const TIn*)q, (const TIn*)k, ws.stats, nullptr, nullptr, dm.M, dm.T, dm.w, chunks,
-                                   dm.scale_log2);
+                                   dm.scale_log2, sl, heads_per_seq);
   lc.mark("score_simt_sweep1");
   score_lse_kernel<<<(unsigned)dm.heads(), 256, 0, st>>>(ws.stats, ws.lse, dm.M, chunks);
   lc.mark("score_lse");
   k2<<<grid, kThreads, smem, st>>>((const TIn*)q, (const TIn*)k, nullptr, ws.lse, ws.raw, dm.M, dm.T, dm.w, chunks,
-                                   dm.scale_log2);
+                                   dm.scale_log2, sl, heads_per_seq);
   lc.mark("score_simt_sweep2");
   return cudaGetLastError();
 }
@@ -261,7 +270,7 @@ cudaError_t launch_lse(const Dims& dm, const float* stats, float* lse, int chunk
 
 cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, HeadRange hr, LaunchCtx& lc) {
   const int half = dm.kp / 2;
-  const bool vec = dm.n % 4 == 0 && half <= 4 && (reinterpret_cast<uintptr_t>(raw) & 15u) == 0 &&
+  const bool vec = !dm.seq_T && dm.n % 4 == 0 && half <= 4 && (reinterpret_cast<uintptr_t>(raw) & 15u) == 0 &&
                    (reinterpret_cast<uintptr_t>(pooled) & 15u) == 0;
   if (vec) {
     const int n4 = dm.n / 4, tiles = (n4 + 255) / 256;
@@ -269,7 +278,11 @@ cudaError_t launch_pool(const Dims& dm, const float* raw, float* pooled, HeadRan
         reinterpret_cast<const float4*>(raw), reinterpret_cast<float4*>(pooled), n4, half, tiles, hr.h0);
   } else {
     const int tiles = (dm.n + 255) / 256;
-    max_pool_kernel<<<(unsigned)((int64_t)hr.nh * tiles), 256, 0, lc.st>>>(raw, pooled, dm.n, half, tiles, hr.h0);
+    SeqLens sl = {};
+    if (dm.seq_T)
+      for (int q = 0; q < dm.S; ++q) sl.T[q] = dm.seq_T[q];
+    max_pool_kernel<<<(unsigned)((int64_t)hr.nh * tiles), 256, 0, lc.st>>>(raw, pooled, dm.n, half, tiles, hr.h0, sl,
+                                                                           dm.seq_T ? dm.N : 0, dm.w);
   }
   lc.mark("max_pool");
   return cudaGetLastError();

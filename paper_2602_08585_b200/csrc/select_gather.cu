@@ -36,14 +36,17 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
                                                                 const int32_t* __restrict__ budgets,
                                                                 const int32_t* __restrict__ offsets,
                                                                 int32_t* __restrict__ kept_idx, long long rows_cap,
-                                                                int n, int w, int span_rt, int head0, int n_sink) {
+                                                                int n_stride, int w, int span_rt, int head0, int n_sink,
+                                                                SeqLens sl, int heads_per_seq) {
   __shared__ int hist[2048];
   __shared__ int scan_gt[kSelWarps], scan_eq[kSelWarps];
   __shared__ int sel_digit, sel_want;
   const int u = head0 + blockIdx.x, tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
   const int b = budgets[u];
   const long long off = offsets[u];
-  const float* src = pooled + (size_t)u * n;
+  // n_stride: row stride of the scores (the longest sequence); n: rankable positions of this head's sequence
+  const int n = heads_per_seq > 0 ? sl.T[u / heads_per_seq] - w : n_stride;
+  const float* src = pooled + (size_t)u * n_stride;
   int32_t* out = kept_idx + off;
   const long long room = rows_cap - off;  // rows of this head that fit in the output
 
@@ -274,20 +277,24 @@ cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* bu
   cudaStream_t st = lc.st;
   const unsigned grid = (unsigned)hr.nh;
   const int n = dm.n;
+  SeqLens sl = {};
+  const int hps = dm.seq_T ? dm.N : 0;
+  if (dm.seq_T)
+    for (int q = 0; q < dm.S; ++q) sl.T[q] = dm.seq_T[q];
   if (n <= kSelThreads * 2)
     select_kernel<2><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
-                                                    dm.n_sink);
+                                                    dm.n_sink, sl, hps);
   else if (n <= kSelThreads * 8)
     select_kernel<8><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
-                                                    dm.n_sink);
+                                                    dm.n_sink, sl, hps);
   else if (n <= kSelThreads * 32)
     select_kernel<32><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
-                                                    dm.n_sink);
+                                                    dm.n_sink, sl, hps);
   else {
     const int per_warp = (n + kSelWarps - 1) / kSelWarps;
     const int span = (per_warp + 31) & ~31;
     select_kernel<0><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, span, hr.h0,
-                                                   dm.n_sink);
+                                                   dm.n_sink, sl, hps);
   }
   lc.mark("select");
   return cudaGetLastError();

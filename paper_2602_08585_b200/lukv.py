@@ -23,7 +23,8 @@ DTYPE_BF16, DTYPE_FP32 = 0, 1
 EXPORTS = ("lukv_workspace_bytes", "lukv_score", "lukv_allocate", "lukv_select_gather", "lukv_compress",
            "lukv_strerror", "lukv_last_launch_count", "lukv_compress_profile", "lukv_allocate_static",
            "lukv_profile_workspace_bytes", "lukv_profile_build", "lukv_profile_budgets", "lukv_build_curves", "lukv_exact_workspace_bytes",
-           "lukv_exact_allocate", "lukv_importance_workspace_bytes", "lukv_oracle_importance")
+           "lukv_exact_allocate", "lukv_importance_workspace_bytes", "lukv_oracle_importance", "lukv_score_ragged",
+           "lukv_compress_ragged")
 
 
 class Params(ctypes.Structure):
@@ -84,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.lukv_importance_workspace_bytes.argtypes = [pp, ctypes.c_int32, ctypes.POINTER(sz)]
         L.lukv_oracle_importance.argtypes = [pp, ctypes.c_int32, ctypes.c_int32, vp, vp, vp, vp, vp, ctypes.c_int32, vp,
                                              vp, sz, vp]
+        L.lukv_score_ragged.argtypes = [pp, vp, vp, vp, vp, vp, sz, vp]
+        L.lukv_compress_ragged.argtypes = [pp, vp] + L.lukv_compress.argtypes[1:]
         L.lukv_strerror.argtypes = [ctypes.c_int]
         L.lukv_strerror.restype = ctypes.c_char_p
         for name in EXPORTS[:5] + EXPORTS[6:]:
@@ -253,6 +256,29 @@ def lukv_compress(params: Params, q_win, k, v, curves, budgets_in, k_out, v_out,
                              _ptr(dev_status), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                              _stream(stream))
     return _check(rc, "lukv_compress", check)
+
+
+def _host_lens(ctx_lens) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(ctx_lens, dtype=np.int32))
+
+
+def lukv_score_ragged(params: Params, ctx_lens, q_win, k, scores, ws, stream=None, check: bool = True) -> int:
+    """lukv_score for sequences of different lengths: params.ctx_len is the row stride, ctx_lens [S] host ints."""
+    lens = _host_lens(ctx_lens)
+    rc = lib().lukv_score_ragged(ctypes.byref(params), lens.ctypes.data, _ptr(q_win), _ptr(k), _ptr(scores), _ptr(ws),
+                                 0 if ws is None else ws.numel() * ws.element_size(), _stream(stream))
+    return _check(rc, "lukv_score_ragged", check)
+
+
+def lukv_compress_ragged(params: Params, ctx_lens, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets,
+                         offsets, rows_cap: int, dev_status, ws, stream=None, check: bool = True) -> int:
+    b = _host_budgets(budgets_in)
+    lens = _host_lens(ctx_lens)
+    rc = lib().lukv_compress_ragged(ctypes.byref(params), lens.ctypes.data, _ptr(q_win), _ptr(k), _ptr(v), _ptr(curves),
+                                    b.ctypes.data, _ptr(k_out), _ptr(v_out), _ptr(kept_idx), _ptr(budgets),
+                                    _ptr(offsets), int(rows_cap), _ptr(dev_status), _ptr(ws),
+                                    0 if ws is None else ws.numel() * ws.element_size(), _stream(stream))
+    return _check(rc, "lukv_compress_ragged", check)
 
 
 def lukv_compress_profile(params: Params, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets,

@@ -14,7 +14,7 @@ using namespace lukv;
 
 namespace lukv_bench {
 
-constexpr int kRoleKernel = 0, kRoleSfu = 1, kRolePoly = 2, kRoleMixed = 3;  // mixed: SFU quads beside polynomial quads
+constexpr int kRoleKernel = 0, kRoleSfu = 1, kRolePoly = 2, kRoleMixed = 3, kRoleShfl = 4;  // mixed: SFU quads beside polynomial quads
 constexpr int kMmaLimit = 1 << 22;
 
 __device__ __forceinline__ void sfu_chunk(const float (&v)[32], uint64_t sc2, uint64_t nm2, uint64_t& acc0, uint64_t& acc1) {
@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(512, 1) epilogue_rate(float* out, long long* c
   const uint64_t sc2 = pack2(0.1275f, 0.1275f), nm2 = pack2(-2.f, -2.f);
   uint64_t acc0 = 0ull, acc1 = 0ull;
   float m_run = -INFINITY, l_run = 0.f;
+  const float4 mine4 = *reinterpret_cast<const float4*>(nlse + 4 * lane);
   const int quad = warp >> 2;
   if (quad < q1 + q2) {
     const bool first = quad < q1;
@@ -84,22 +85,24 @@ __global__ void __launch_bounds__(512, 1) epilogue_rate(float* out, long long* c
         tmem_ld_wait(va);
         tmem_ld32(tcol + 32 * (c + 1), vb);
         if (first) {
-          if (ROLE == kRoleKernel) p1_chunk<false>(va, 0, 1 << 30, 0.1275f, m_run, l_run);
+          if (ROLE == kRoleKernel || ROLE == kRoleShfl) p1_chunk<false>(va, 0, 1 << 30, 0.1275f, m_run, l_run);
           else if (ROLE == kRoleSfu || ROLE == kRoleMixed) sfu_chunk(va, sc2, nm2, acc0, acc1);
           else poly_chunk(va, nlse + 32 * c, sc2, acc0, acc1);
         } else {
           if (ROLE == kRoleKernel) p2_chunk(va, nlse + 32 * c, sc2, acc0, acc1);
+          else if (ROLE == kRoleShfl) p2_chunk_shfl(va, mine4, 32 * c, sc2, acc0, acc1);
           else if (ROLE == kRoleSfu) sfu_chunk(va, sc2, nm2, acc0, acc1);
           else poly_chunk(va, nlse + 32 * c, sc2, acc0, acc1);
         }
         tmem_ld_wait(vb);
         if (c + 2 < 4) tmem_ld32(tcol + 32 * (c + 2), va);
         if (first) {
-          if (ROLE == kRoleKernel) p1_chunk<false>(vb, 0, 1 << 30, 0.1275f, m_run, l_run);
+          if (ROLE == kRoleKernel || ROLE == kRoleShfl) p1_chunk<false>(vb, 0, 1 << 30, 0.1275f, m_run, l_run);
           else if (ROLE == kRoleSfu || ROLE == kRoleMixed) sfu_chunk(vb, sc2, nm2, acc0, acc1);
           else poly_chunk(vb, nlse + 32 * (c + 1), sc2, acc0, acc1);
         } else {
           if (ROLE == kRoleKernel) p2_chunk(vb, nlse + 32 * (c + 1), sc2, acc0, acc1);
+          else if (ROLE == kRoleShfl) p2_chunk_shfl(vb, mine4, 32 * (c + 1), sc2, acc0, acc1);
           else if (ROLE == kRoleSfu) sfu_chunk(vb, sc2, nm2, acc0, acc1);
           else poly_chunk(vb, nlse + 32 * (c + 1), sc2, acc0, acc1);
         }
@@ -259,6 +262,8 @@ int main() {
   for (int q = 1; q <= 3; ++q) run_case<kRoleKernel>("kernel's chunk functions", 0, q, 0, out, clk, sms, tiles);
   run_case<kRoleKernel>("kernel's chunk functions", 2, 0, 1, out, clk, sms, tiles);
   run_case<kRoleKernel>("kernel's chunk functions", 0, 2, 1, out, clk, sms, tiles);
+  run_case<kRoleShfl>("pass 2, -lse by shuffles", 0, 2, 0, out, clk, sms, tiles);
+  run_case<kRoleShfl>("pass 2, -lse by shuffles", 0, 2, 1, out, clk, sms, tiles);
   run_case<kRoleKernel>("kernel's chunk functions", 1, 1, 0, out, clk, sms, tiles);
   run_case<kRoleKernel>("kernel's chunk functions", 1, 1, 1, out, clk, sms, tiles);
   for (int q = 1; q <= 3; ++q) run_case<kRoleSfu>("exp2 on the SFU only", q, 0, 0, out, clk, sms, tiles);

@@ -149,3 +149,36 @@ def test_compress_batch_is_per_sequence(oracle):
         np.testing.assert_array_equal(out["kept_idx"][lo:hi], single["kept_idx"])
         np.testing.assert_array_equal(out["k_out"][lo:hi], single["k_out"])
         np.testing.assert_array_equal(out["budgets"][s_], single["budgets"][0])
+
+
+def test_ragged_batch_is_the_concatenation_of_single_sequence_runs(oracle):
+    O = oracle
+    """Sequences of different lengths in one batch (App. E): by definition one run per sequence.  With equal
+    lengths the ragged form must reproduce the batched run bit for bit; with different lengths every sequence
+    must be untouched by its neighbours and by the padding behind its last position."""
+    rng = np.random.default_rng(12)
+    S, L, H, G, d, T, w, kp, P = 3, 1, 2, 2, 8, 48, 4, 3, 9
+    q = rng.standard_normal((S, L, H * G, w, d)).astype(np.float32)
+    k = rng.standard_normal((S, L, H, T, d)).astype(np.float32)
+    v = rng.standard_normal((S, L, H, T, d)).astype(np.float32)
+    U = np.zeros((L * H, P), np.float32)
+    U[:, 1:] = np.cumsum(rng.exponential(size=(L * H, P - 1)), axis=1)
+    same = O.compress_ragged(q, k, v, U, [20, 31, 7], [T, T, T], G, kp)
+    ref = O.compress(q, k, v, U, [20, 31, 7], G, kp)
+    for key in ("k_out", "v_out", "kept_idx", "budgets", "offsets"):
+        np.testing.assert_array_equal(same[key], ref[key])
+    lens = [48, 32, 16]                       # each a multiple of P-1 = 8
+    rag = O.compress_ragged(q, k, v, U, [20, 15, 7], lens, G, kp)
+    k2, v2 = k.copy(), v.copy()
+    k2[1, :, :, 32:] = 99.0                   # padding behind a sequence's last position is never read
+    v2[2, :, :, 16:] = -99.0
+    rag2 = O.compress_ragged(q, k2, v2, U, [20, 15, 7], lens, G, kp)
+    for key in ("k_out", "v_out", "kept_idx", "budgets", "offsets"):
+        np.testing.assert_array_equal(rag[key], rag2[key])
+    assert rag["offsets"][-1] == 20 + 15 + 7 + S * L * H * w
+    for s, Ts in enumerate(lens):
+        one = O.compress(q[s:s + 1], k[s:s + 1, :, :, :Ts], v[s:s + 1, :, :, :Ts], U, [[20, 15, 7][s]], G, kp)
+        np.testing.assert_array_equal(rag["budgets"][s], one["budgets"][0])
+        r0, r1 = rag["offsets"][s * L * H], rag["offsets"][(s + 1) * L * H]
+        np.testing.assert_array_equal(rag["kept_idx"][r0:r1], one["kept_idx"])
+        assert rag["kept_idx"][r0:r1].max() == Ts - 1          # the window ends at the sequence's own last position
