@@ -39,9 +39,10 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_32k",
                     help="a configuration name, or 'all': one JSON line per configuration (single GPU)")
-    ap.add_argument("--path", default="compress", choices=["compress", "profile"],
+    ap.add_argument("--path", default="compress", choices=["compress", "profile", "ragged"],
                     help="compress: the headline path; profile: the offline profile build and the online "
-                         "lookup front end (secondary measurement, single GPU)")
+                         "lookup front end; ragged: a batch of different context lengths in one call against one "
+                         "call per sequence (secondary measurements, single GPU)")
     ap.add_argument("--sinks", type=int, default=0, help="attention sinks kept in every head (App. E uses 4)")
     ap.add_argument("--min-keep", type=float, default=0.0,
                     help="minimum retention per head (App. E uses 0.01); default off, as the headline "
@@ -604,6 +605,85 @@ def run_profile_path(args):
         "clocks": sampler.summary(), "cpu_baseline": cpu}))
 
 
+def run_ragged_path(args):
+    """Secondary measurement (App. E deployment): the batch of configuration 4 with eight different context
+    lengths, compressed by one lukv_compress_ragged call and, for comparison, by one lukv_compress call per
+    sequence on the same padded cache."""
+    import torch
+    from paper_2602_08585_b200 import lukv, synth
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (the path has no CPU fallback)"
+    torch.cuda.set_device(0)
+    lukv.lib()
+    wl = synth.CONFIGS["batch8_16k_mixed"]
+    if args.layers > 0:
+        wl = synth.scaled(wl, L=args.layers, name=f"{wl.name}[layers={args.layers}]")
+    fr = [1.0, 0.5, 0.75, 0.25, 0.875, 0.375, 0.625, 0.125]
+    lens = [int(wl.T * fr[q % len(fr)]) for q in range(wl.S)]         # multiples of T/8, hence of the curve grid
+    p = lukv.make_params(wl.S, wl.L, wl.H, wl.G, wl.d, wl.T, wl.w, wl.kp, wl.dtype, wl.P)
+    q, k, v = synth.gen_tensors(wl, "cuda")
+    curves = torch.from_numpy(synth.gen_curves(wl)).cuda()
+    Bs = [int(wl.keep[i % len(wl.keep)] * wl.N * (lens[i] - wl.w)) for i in range(wl.S)]
+    ws = lukv.alloc_workspace(p)
+    out = lukv.Outputs(p, Bs)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    def one_call():
+        lukv.lukv_compress_ragged(p, lens, q, k, v, curves, Bs, out.k_out, out.v_out, out.kept_idx, out.budgets,
+                                  out.offsets, out.rows, out.dev_status, ws)
+
+    ragged_ms = timed(one_call)
+    launches = lukv.lukv_last_launch_count()
+    assert int(out.dev_status.item()) == 0
+    kept_ragged = out.kept_idx.clone()
+
+    # one call per sequence: the sequence's own parameters on contiguous copies of its part of the cache
+    per = []
+    row0 = 0
+    for i in range(wl.S):
+        pi = lukv.make_params(1, wl.L, wl.H, wl.G, wl.d, lens[i], wl.w, wl.kp, wl.dtype, wl.P)
+        ki = k[i:i + 1, :, :, :lens[i]].contiguous()
+        vi = v[i:i + 1, :, :, :lens[i]].contiguous()
+        oi = lukv.Outputs(pi, Bs[i:i + 1])
+        per.append((pi, q[i:i + 1], ki, vi, oi, lukv.alloc_workspace(pi), row0))
+        row0 += oi.rows
+    launches_per_seq = []
+
+    def per_sequence():
+        launches_per_seq.clear()
+        for pi, qi, ki, vi, oi, wsi, _ in per:
+            lukv.lukv_compress(pi, qi, ki, vi, curves, [int(oi.rows - wl.N * wl.w)], oi.k_out, oi.v_out, oi.kept_idx,
+                               oi.budgets, oi.offsets, oi.rows, oi.dev_status, wsi)
+            launches_per_seq.append(lukv.lukv_last_launch_count())
+
+    seq_ms = timed(per_sequence)
+    same = sum(int((kept_ragged[r0:r0 + oi.rows] == oi.kept_idx).sum().item()) for *_, oi, _w, r0 in per)
+    tokens = sum(lens)
+    es = 2 if wl.dtype == "bf16" else 4
+    print(json.dumps({
+        "metric": METRIC, "value": tokens / (ragged_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ragged_ms, "higher_is_better": True, "vs_baseline": None,
+        "dtype": "bf16 in / f32 accumulate", "data": "synthetic (seeded)",
+        "config": {"workload": f"ragged[{wl.name}]", "ctx_lens": lens, "layers": wl.L, "kv_heads": wl.H,
+                   "packed_rows": out.rows, "row_stride_T": wl.T},
+        "gpu_launches": launches * args.steps,
+        "one_call_per_sequence": {"ms_per_step": seq_ms, "launches_per_step": sum(launches_per_seq),
+                                  "kept_rows_identical_to_the_ragged_call": same, "kept_rows": out.rows},
+        "launches_per_step": launches,
+        "path_bytes_per_step": tokens * wl.N * wl.d * es + 2 * out.rows * wl.d * es}))
+
+
 def pick_workload(args):
     from paper_2602_08585_b200 import synth
     wl = synth.CONFIGS[args.workload]
@@ -619,6 +699,9 @@ def main():
     elif args.path == "profile":
         if int(os.environ.get("RANK", "0")) == 0:
             run_profile_path(args)
+    elif args.path == "ragged":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_ragged_path(args)
     elif args.workload == "all":
         # one line per configuration, each with its own roofline and clocks (single GPU; the end-to-end and CPU
         # legs only for the headline configuration)
