@@ -26,6 +26,10 @@
 //              a cached position makes to the head output over K_max decode steps, attention weight
 //              times the L2 norm of the projected value (App. E names the norm and an intra-layer
 //              normalisation); readings for grouped queries and the normalisation in the design notes.
+//   keydiff  : the second proxy metric the paper evaluates (Sec. 5.1, pi_2; App. E: recent window 1).  The paper
+//              only names it ("the geometric features of key vectors"); the formula restated here is the one of
+//              the method's own publication (a key's score is the negated cosine similarity between the key and
+//              the mean of all unit-normalised keys of its head), recorded as a reading in the design notes.
 //   exact    : the allocation problem on the raw curves by the multiple-choice-knapsack
 //              recursion (Sec. 4.2 mentions the exact solver as the comparison point).
 //   deployment settings (App. E): attention sinks always ranked first; a minimum number of
@@ -46,7 +50,9 @@
 // search, against the greedy on concave curves, and between the greedy's raw and hull values;
 // the oracle importance against a library softmax times a library vector norm (one decode step,
 // identity projection), closed forms for identical keys, monotonicity in K_max, a dominant decode
-// key, doubling under two identical grouped query heads, and unit mass per layer after normalisation.
+// key, doubling under two identical grouped query heads, and unit mass per layer after normalisation;
+// the KeyDiff score against library cosine-similarity and normalisation routines, closed forms
+// (identical keys, one odd key out, two opposite groups), and invariance to rescaling single keys.
 // No function here is "parity unpinned".
 //
 // Build: g++ -O2 -std=c++17 -ffp-contract=off -shared -fPIC lukv_oracle.cpp -o liblukv_oracle.so
@@ -530,6 +536,41 @@ void oracle_importance(const void* q_dec, const void* k, const void* v, const vo
       }
   }
   for (size_t i = 0; i < imp.size(); ++i) importance[i] = to_f32_ftz(imp[i]);
+}
+
+
+// KeyDiff proxy (pi_2 of Sec. 5.1; formula from the method's own publication, see the header):
+//   u_j = k_j / max(||k_j||, eps),   a = (1/T) sum_{j<T} u_j   (all T cached keys of the head, window included),
+//   score_j = - <k_j, a> / (max(||k_j||, eps) * max(||a||, eps)),   eps = 1e-8,   for the n = T-w rankable positions.
+// Keys far from the head's mean key direction score high and are kept.  k [heads][T][d]; out [heads][T-w] fp32.
+void oracle_keydiff(const void* k, int dtype, int heads, int T, int w, int d, float* scores) {
+  const int n = T - w;
+  const double eps = 1e-8;
+  std::vector<double> anchor(d), norm(T);
+  for (int u = 0; u < heads; ++u) {
+    const int64_t base = static_cast<int64_t>(u) * T * d;
+    std::fill(anchor.begin(), anchor.end(), 0.0);
+    for (int j = 0; j < T; ++j) {
+      double ss = 0.0;
+      for (int c = 0; c < d; ++c) {
+        const double x = load_elem(k, dtype, base + static_cast<int64_t>(j) * d + c);
+        ss += x * x;
+      }
+      norm[j] = std::max(std::sqrt(ss), eps);
+      for (int c = 0; c < d; ++c) anchor[c] += load_elem(k, dtype, base + static_cast<int64_t>(j) * d + c) / norm[j];
+    }
+    double an = 0.0;
+    for (int c = 0; c < d; ++c) {
+      anchor[c] /= static_cast<double>(T);
+      an += anchor[c] * anchor[c];
+    }
+    an = std::max(std::sqrt(an), eps);
+    for (int j = 0; j < n; ++j) {
+      double dot = 0.0;
+      for (int c = 0; c < d; ++c) dot += load_elem(k, dtype, base + static_cast<int64_t>(j) * d + c) * anchor[c];
+      scores[static_cast<int64_t>(u) * n + j] = static_cast<float>(-dot / (norm[j] * an));
+    }
+  }
 }
 
 

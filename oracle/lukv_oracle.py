@@ -268,6 +268,16 @@ def importance(q_dec, k, v, w_o, G: int, w: int, k_dec=None, scale: float = 0.0,
     return out
 
 
+def keydiff(k, w: int) -> np.ndarray:
+    """KeyDiff proxy scores: k [S][L][H][T][d] -> [S][L*H][T-w] float32 (negated cosine similarity of every
+    rankable key with the mean of the head's unit-normalised keys)."""
+    k = _c(k)
+    S, L, H, T, d = k.shape
+    out = np.empty((S, L * H, T - w), np.float32)
+    lib().oracle_keydiff(_p(k), _dtype_code(k), S * L * H, T, w, d, _p(out))
+    return out
+
+
 def exact_allocate(curves, T: int, w: int, budgets_in):
     """Exact allocation on token-resolution curves [N][T+1] -> (budgets [S][N] int32, optimum values [S] float64)."""
     curves = _c(curves, np.float32)
