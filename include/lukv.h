@@ -114,6 +114,22 @@ LUKV_API int lukv_score(const lukv_params_t* params, const void* q_win, const vo
                size_t ws_bytes, void* stream);
 
 /*
+ * Stage (a) with the second proxy metric the paper evaluates, KeyDiff (pi_2 of Sec. 5.1; App. E uses a recent
+ * window of 1 with it).  The paper only names the metric ("the geometric features of key vectors"); the formula
+ * implemented is the one of the method's own publication: with u_j = k_j / max(||k_j||, eps) and the anchor
+ * a = mean of u_j over all T cached keys of the head,
+ *     scores[j] = - <k_j, a> / (max(||k_j||, eps) * max(||a||, eps)),   eps = 1e-8,
+ * for the n = T-w rankable positions: keys far from the head's mean key direction score high and are kept first.
+ * No queries, no pooling (pool_kernel must be valid but is unused).  The scores lie in [-1, 1]; they feed
+ * lukv_select_gather and lukv_build_curves like the scores of lukv_score.
+ *
+ *   k      [S][L][H][T][d]
+ *   scores [S][N][n] fp32     out
+ */
+LUKV_API int lukv_score_keydiff(const lukv_params_t* params, const void* k, float* scores, void* ws, size_t ws_bytes,
+                                void* stream);
+
+/*
  * Stage (b): global head-level budget allocation (Sec. 4.2; App. A.2).
  * (b1) Hull relaxation: the P-1 increments of each head's utility curve are projected by
  *      pool-adjacent-violators onto a non-increasing sequence and clipped at 0
@@ -145,7 +161,7 @@ LUKV_API int lukv_allocate(const lukv_params_t* params, const float* curves, con
  *   kept_idx[o+b .. o+b+w)  the window positions n .. T-1
  *   k_out / v_out row r     = k / v row kept_idx[r] of head u, copied bit for bit
  *
- *   scores   [S][N][n] fp32   pooled scores (non-negative, finite)
+ *   scores   [S][N][n] fp32   scores of the rankable positions (finite; any sign)
  *   budgets  [S][N] int32, offsets [S*N+1] int32   as produced by lukv_allocate; the
  *            caller guarantees 0 <= budgets <= n and offsets consistent with them
  *   k, v     [S][L][H][T][d]

@@ -29,6 +29,7 @@ Workspace carve_workspace(const Dims& dm, void* base) {
   size_t stats_bytes = score_tc_stats_bytes(dm);
   if (stats_simt > stats_bytes) stats_bytes = stats_simt;
   if (score_onepass_stats_bytes(dm) > stats_bytes) stats_bytes = score_onepass_stats_bytes(dm);
+  if (keydiff_scratch_bytes(dm) > stats_bytes) stats_bytes = keydiff_scratch_bytes(dm);
   ws.stats = static_cast<float*>(take(stats_bytes));
   ws.lse = static_cast<float*>(take(heads * dm.M * sizeof(float)));
   ws.gains = static_cast<float*>(take((size_t)dm.N * (dm.P - 1) * sizeof(float)));
@@ -240,6 +241,21 @@ int lukv_score(const lukv_params_t* params, const void* q_win, const void* k, fl
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;
   if (run_score(dm, q_win, k, w, scores, nullptr, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  g_last_launches = lc.launches;
+  return LUKV_OK;
+}
+
+int lukv_score_keydiff(const lukv_params_t* params, const void* k, float* scores, void* ws, size_t ws_bytes,
+                       void* stream) {
+  Dims dm;
+  int rc = make_dims(params, &dm);
+  if (rc != LUKV_OK) return rc;
+  if (!k || !scores || !aligned16(k)) return LUKV_ERR_INVALID_ARG;
+  Workspace w;
+  if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
+  LaunchCtx lc;
+  lc.st = (cudaStream_t)stream;
+  if (launch_keydiff(dm, k, scores, w.stats, lc) != cudaSuccess) return LUKV_ERR_CUDA;
   g_last_launches = lc.launches;
   return LUKV_OK;
 }

@@ -129,6 +129,9 @@ cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, cons
 size_t curves_smem_bytes(int n, int P);
 cudaError_t launch_build_curves(const Dims& dm, const float* scores, const float* importance, float* curves,
                                 LaunchCtx& lc);
+// KeyDiff proxy scores (key-only metric): scores [heads][n]; scratch of keydiff_scratch_bytes().
+size_t keydiff_scratch_bytes(const Dims& dm);
+cudaError_t launch_keydiff(const Dims& dm, const void* k, float* scores, float* scratch, LaunchCtx& lc);
 // Oracle importance of Sec. 4.1 from decode queries, the cache and the output projection.
 size_t importance_workspace_bytes(const Dims& dm, int k_max);
 cudaError_t launch_importance(const Dims& dm, int k_max, int d_model, const void* q_dec, const void* k, const void* v,
