@@ -123,11 +123,14 @@ LUKV_API int lukv_score(const lukv_params_t* params, const void* q_win, const vo
  * No queries, no pooling (pool_kernel must be valid but is unused).  The scores lie in [-1, 1]; they feed
  * lukv_select_gather and lukv_build_curves like the scores of lukv_score.
  *
- *   k      [S][L][H][T][d]
- *   scores [S][N][n] fp32     out
+ *   k          [S][L][H][T][d]
+ *   scores     [S][N][n] fp32     out
+ *   dev_status [1] int32, may be NULL: set to 0 by the call; LUKV_ERR_TIMEOUT if a bounded wait ran out (the
+ *              kernel's CTAs wait for one another's partial sums of a head; it is launched cooperatively, so
+ *              this only happens if the device is taken away).  The scores are then undefined.
  */
-LUKV_API int lukv_score_keydiff(const lukv_params_t* params, const void* k, float* scores, void* ws, size_t ws_bytes,
-                                void* stream);
+LUKV_API int lukv_score_keydiff(const lukv_params_t* params, const void* k, float* scores, int32_t* dev_status, void* ws,
+                       size_t ws_bytes, void* stream);
 
 /*
  * Stage (b): global head-level budget allocation (Sec. 4.2; App. A.2).

@@ -245,8 +245,8 @@ int lukv_score(const lukv_params_t* params, const void* q_win, const void* k, fl
   return LUKV_OK;
 }
 
-int lukv_score_keydiff(const lukv_params_t* params, const void* k, float* scores, void* ws, size_t ws_bytes,
-                       void* stream) {
+int lukv_score_keydiff(const lukv_params_t* params, const void* k, float* scores, int32_t* dev_status, void* ws,
+                       size_t ws_bytes, void* stream) {
   Dims dm;
   int rc = make_dims(params, &dm);
   if (rc != LUKV_OK) return rc;
@@ -255,7 +255,8 @@ int lukv_score_keydiff(const lukv_params_t* params, const void* k, float* scores
   if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;
-  if (launch_keydiff(dm, k, scores, w.stats, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (dev_status && cudaMemsetAsync(dev_status, 0, sizeof(int32_t), lc.st) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (launch_keydiff(dm, k, scores, w.stats, dev_status, lc) != cudaSuccess) return LUKV_ERR_CUDA;
   g_last_launches = lc.launches;
   return LUKV_OK;
 }

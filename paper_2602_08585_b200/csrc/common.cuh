@@ -131,7 +131,8 @@ cudaError_t launch_build_curves(const Dims& dm, const float* scores, const float
                                 LaunchCtx& lc);
 // KeyDiff proxy scores (key-only metric): scores [heads][n]; scratch of keydiff_scratch_bytes().
 size_t keydiff_scratch_bytes(const Dims& dm);
-cudaError_t launch_keydiff(const Dims& dm, const void* k, float* scores, float* scratch, LaunchCtx& lc);
+cudaError_t launch_keydiff(const Dims& dm, const void* k, float* scores, float* scratch, int32_t* dev_status,
+                           LaunchCtx& lc);
 // Oracle importance of Sec. 4.1 from decode queries, the cache and the output projection.
 size_t importance_workspace_bytes(const Dims& dm, int k_max);
 cudaError_t launch_importance(const Dims& dm, int k_max, int d_model, const void* q_dec, const void* k, const void* v,

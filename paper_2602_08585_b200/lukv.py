@@ -86,7 +86,7 @@ def lib() -> ctypes.CDLL:
         L.lukv_oracle_importance.argtypes = [pp, ctypes.c_int32, ctypes.c_int32, vp, vp, vp, vp, vp, ctypes.c_int32, vp,
                                              vp, sz, vp]
         L.lukv_score_ragged.argtypes = [pp, vp, vp, vp, vp, vp, sz, vp]
-        L.lukv_score_keydiff.argtypes = [pp, vp, vp, vp, sz, vp]
+        L.lukv_score_keydiff.argtypes = [pp, vp, vp, vp, vp, sz, vp]
         L.lukv_compress_ragged.argtypes = [pp, vp] + L.lukv_compress.argtypes[1:]
         L.lukv_strerror.argtypes = [ctypes.c_int]
         L.lukv_strerror.restype = ctypes.c_char_p
@@ -259,9 +259,9 @@ def lukv_compress(params: Params, q_win, k, v, curves, budgets_in, k_out, v_out,
     return _check(rc, "lukv_compress", check)
 
 
-def lukv_score_keydiff(params: Params, k, scores, ws, stream=None, check: bool = True) -> int:
-    """KeyDiff proxy scores: k [S][L][H][T][d] -> scores [S][N][n] fp32 (device)."""
-    rc = lib().lukv_score_keydiff(ctypes.byref(params), _ptr(k), _ptr(scores), _ptr(ws),
+def lukv_score_keydiff(params: Params, k, scores, ws, dev_status=None, stream=None, check: bool = True) -> int:
+    """KeyDiff proxy scores: k [S][L][H][T][d] -> scores [S][N][n] fp32 (device); dev_status [1] int32 or None."""
+    rc = lib().lukv_score_keydiff(ctypes.byref(params), _ptr(k), _ptr(scores), _ptr(dev_status), _ptr(ws),
                                   0 if ws is None else ws.numel() * ws.element_size(), _stream(stream))
     return _check(rc, "lukv_score_keydiff", check)
 

@@ -1,7 +1,7 @@
 """GPU parity of the KeyDiff proxy (pi_2 of Sec. 5.1) against the oracle, and the path built on it: KeyDiff scores
 -> per-head top-b selection and gather with the recent window of 1 that App. E uses for this metric.
 The scores are cosines in [-1, 1] from fp32 sums over d channels and T keys: absolute tolerance 2e-5 (the anchor
-is a mean of T unit vectors accumulated in fp32 in chunks of 512; the dot products add d terms)."""
+is a mean of T unit vectors accumulated in fp32 in slices of a few hundred keys; the dot products add d terms)."""
 import numpy as np
 import pytest
 import torch
@@ -16,8 +16,10 @@ ATOL = 2e-5
 def gpu_keydiff(p, k):
     ws = lukv.alloc_workspace(p)
     scores = torch.full((p.batch, p.N, p.n), -7.0, dtype=torch.float32, device="cuda")
-    lukv.lukv_score_keydiff(p, k.cuda(), scores, ws)
+    status = torch.full((1,), 5, dtype=torch.int32, device="cuda")
+    lukv.lukv_score_keydiff(p, k.cuda(), scores, ws, status)
     torch.cuda.synchronize()
+    assert int(status.item()) == 0
     return scores
 
 
@@ -29,6 +31,8 @@ SHAPES = [
     (1, 1, 2, 128, 1025, 5, torch.float32),        # 32 lanes per key row, wider window
     (1, 1, 3, 64, 4096 + 33, 33, torch.float32),
     (1, 4, 8, 128, 16384, 1, torch.bfloat16),      # more heads than one L2 group of keys holds at this length
+    (2, 4, 8, 64, 300, 7, torch.bfloat16),         # many short heads: slices that span several heads
+    (1, 2, 5, 128, 64 * 37 + 1, 1, torch.float32), # one row past a whole number of stages
 ]
 
 
@@ -43,6 +47,47 @@ def test_keydiff_matches_oracle(oracle, shape):
     ref = oracle.keydiff(bits(k), w)
     np.testing.assert_allclose(got, ref, rtol=0, atol=ATOL)
     assert got[0, 0, 0] == 0.0
+
+
+@pytest.mark.parametrize("group_mb", [1, 2, 3])
+def test_keydiff_many_groups(oracle, monkeypatch, group_mb):
+    """Groups of one to three heads (the group size is a tuning switch): every CTA alternates many times between
+    summing one group and scoring the one before it, and the last group is smaller than the others."""
+    monkeypatch.setenv("LUKV_KEYDIFF_GROUP_MB", str(group_mb))
+    S, L, H, d, T, w = 1, 1, 7, 128, 4096, 1          # 1 MB of bf16 keys per head
+    g = torch.Generator().manual_seed(group_mb)
+    k = (torch.randn((S, L, H, T, d), generator=g) + 0.5).to(torch.bfloat16)
+    p = lukv.make_params(S, L, H, 1, d, T, w, 1, torch.bfloat16, 2)
+    got = gpu_keydiff(p, k).cpu().numpy()
+    np.testing.assert_allclose(got, oracle.keydiff(bits(k), w), rtol=0, atol=ATOL)
+
+
+def test_keydiff_wait_runs_out(monkeypatch):
+    """A head whose anchor is never published (a host-side switch of the library drops the publication): the CTAs
+    that score it give up after the bounded wait, the call reports LUKV_ERR_TIMEOUT in dev_status, the device stays
+    usable and the next call is correct."""
+    S, L, H, d, T, w = 1, 1, 4, 128, 2048, 1
+    g = torch.Generator().manual_seed(5)
+    k = torch.randn((S, L, H, T, d), generator=g).to(torch.bfloat16).cuda()
+    p = lukv.make_params(S, L, H, 1, d, T, w, 1, torch.bfloat16, 2)
+    ws = lukv.alloc_workspace(p)
+    scores = torch.empty((S, L * H, T - w), dtype=torch.float32, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+
+    def call():
+        lukv.lukv_score_keydiff(p, k, scores, ws, status)
+        torch.cuda.synchronize()
+        return int(status.item())
+
+    assert call() == 0
+    good = scores.clone()
+    monkeypatch.setenv("LUKV_TEST_SPIN_LIMIT", "20000")
+    monkeypatch.setenv("LUKV_TEST_DROP_ITEM", "2")
+    assert call() == lukv.ERR_TIMEOUT
+    monkeypatch.delenv("LUKV_TEST_SPIN_LIMIT")
+    monkeypatch.delenv("LUKV_TEST_DROP_ITEM")
+    assert call() == 0
+    assert torch.equal(scores, good)
 
 
 def test_keydiff_selection_and_gather(oracle):
