@@ -115,8 +115,8 @@ LUKV_API int lukv_score(const lukv_params_t* params, const void* q_win, const vo
 
 /*
  * Stage (a) with the second proxy metric the paper evaluates, KeyDiff (pi_2 of Sec. 5.1; App. E uses a recent
- * window of 1 with it).  The paper only names the metric ("the geometric features of key vectors"); the formula
- * implemented is the one of the method's own publication: with u_j = k_j / max(||k_j||, eps) and the anchor
+ * window of 1 with it).  The paper only names the metric (as one that looks at the geometry of the key vectors);
+ * the formula implemented is the one of the method's own publication: with u_j = k_j / max(||k_j||, eps) and the anchor
  * a = mean of u_j over all T cached keys of the head,
  *     scores[j] = - <k_j, a> / (max(||k_j||, eps) * max(||a||, eps)),   eps = 1e-8,
  * for the n = T-w rankable positions: keys far from the head's mean key direction score high and are kept first.

@@ -27,7 +27,7 @@
 //              times the L2 norm of the projected value (App. E names the norm and an intra-layer
 //              normalisation); readings for grouped queries and the normalisation in the design notes.
 //   keydiff  : the second proxy metric the paper evaluates (Sec. 5.1, pi_2; App. E: recent window 1).  The paper
-//              only names it ("the geometric features of key vectors"); the formula restated here is the one of
+//              only names it (as a metric on the geometry of the key vectors); the formula restated here is the one of
 //              the method's own publication (a key's score is the negated cosine similarity between the key and
 //              the mean of all unit-normalised keys of its head), recorded as a reading in the design notes.
 //   exact    : the allocation problem on the raw curves by the multiple-choice-knapsack
