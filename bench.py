@@ -534,7 +534,21 @@ def run_profile_path(args):
     keydiff_k_bytes = kk.numel() * kk.element_size()
     keydiff_bytes = keydiff_k_bytes + kd_out.numel() * 4
     assert int(kd_status.item()) == 0, "the KeyDiff kernel gave up on a bounded wait"
-    del kk, kd_ws, kd_out
+    del kd_ws, kd_out
+    # the whole path with KeyDiff as the proxy metric (recent window 1, no pooling), same curves and keep ratio
+    pkp = lukv.make_params(wl.S, wl.L, wl.H, 1, wl.d, wl.T, 1, 1, wl.dtype, wl.P, flags=lukv.FLAG_KEYDIFF)
+    kd_Bs = [int(b * (wl.T - 1) // (wl.T - wl.w)) for b in wl.budgets()]
+    kd_curves = torch.from_numpy(synth.gen_curves(wl)).cuda()
+    kd_vv = torch.randn((wl.S, wl.L, wl.H, wl.T, wl.d), generator=g, device="cuda").to(dt)
+    kd_ws = lukv.alloc_workspace(pkp)
+    kd_o = lukv.Outputs(pkp, kd_Bs)
+    kd_path_ms = timed(lambda: lukv.lukv_compress(pkp, None, kk, kd_vv, kd_curves, kd_Bs, kd_o.k_out, kd_o.v_out,
+                                                  kd_o.kept_idx, kd_o.budgets, kd_o.offsets, kd_o.rows,
+                                                  kd_o.dev_status, kd_ws), args.steps, 3)
+    kd_path_launches = lukv.lukv_last_launch_count()
+    assert int(kd_o.dev_status.item()) == 0
+    kd_rows = kd_o.rows
+    del kk, kd_vv, kd_ws, kd_o, kd_curves
 
     build_ms = timed(lambda: lukv.lukv_profile_build(calib, U, Mq, ratios, phi, pws), args.steps, max(args.warmup, 3))
     build_launches = lukv.lukv_last_launch_count()
@@ -614,6 +628,9 @@ def run_profile_path(args):
         "keydiff_scores": {"ms_per_call": keydiff_ms, "launches": keydiff_launches,
                            "algorithmic_bytes": keydiff_bytes, "gbs": keydiff_bytes / (keydiff_ms * 1e-3) / 1e9,
                            "frac_of_measured_hbm_peak": keydiff_bytes / (keydiff_ms * 1e-3) / 1e9 / measured_peak()[0],
+                           "whole_path": {"metric": METRIC, "value": wl.S * wl.T / (kd_path_ms * 1e-3), "unit": UNIT,
+                                          "ms_per_step": kd_path_ms, "launches_per_step": kd_path_launches,
+                                          "packed_rows": kd_rows, "window": 1},
                            "hbm_bytes_by_design": keydiff_k_bytes + keydiff_bytes,
                            "frac_by_design": (keydiff_k_bytes + keydiff_bytes) / (keydiff_ms * 1e-3) / 1e9
                                              / measured_peak()[0]},

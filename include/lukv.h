@@ -50,7 +50,7 @@ extern "C" {
 
 typedef enum lukv_status {
   LUKV_OK = 0,
-  LUKV_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, flags != 0           */
+  LUKV_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, unknown flag bits     */
   LUKV_ERR_UNSUPPORTED = -2,         /* d not in {64,128}, unknown dtype, even kp, (P-1) does  */
                                      /* not divide T, G*w > 256, P > 4097, N > 18944, sizes    */
                                      /* beyond int32                                           */
@@ -63,6 +63,15 @@ typedef enum lukv_status {
 } lukv_status;
 
 enum { LUKV_DTYPE_BF16 = 0, LUKV_DTYPE_FP32 = 1 };
+
+/*
+ * lukv_params_t.flags.  LUKV_FLAG_KEYDIFF: the proxy metric of stage (a) is KeyDiff (see lukv_score_keydiff)
+ * instead of the observation-window attention scores, in lukv_score, lukv_compress and
+ * lukv_compress_profile: q_win is ignored and may be NULL, gqa_group plays no role, pool_kernel must be 1 (the
+ * metric is not pooled); App. E pairs it with window = 1.  The calls for sequences of different lengths return
+ * LUKV_ERR_UNSUPPORTED with this flag.
+ */
+#define LUKV_FLAG_KEYDIFF 1
 
 typedef struct lukv_params {
   int32_t batch;        /* S >= 1                                                             */
@@ -77,7 +86,7 @@ typedef struct lukv_params {
   int32_t dtype;        /* LUKV_DTYPE_BF16 or LUKV_DTYPE_FP32: element type of Q, K and V     */
   int32_t curve_points; /* P, 2 <= P <= 4097, (P-1) divides T                                 */
   float softmax_scale;  /* 0 selects 1/sqrt(d) (Eq. 1)                                        */
-  int32_t flags;        /* reserved, must be 0                                                */
+  int32_t flags;        /* 0, or LUKV_FLAG_KEYDIFF; other bits must be 0                      */
   /* Deployment settings of App. E (implementation details); 0 switches either off.            */
   int32_t n_sink;       /* attention sinks: positions 0..n_sink-1 rank before all others in   */
                         /* the selection whatever their score, so they are kept whenever the  */

@@ -44,7 +44,7 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // must fit every sequence.  On success dm describes the longest sequence and carries the lengths.
 static int attach_seq_lens(Dims* dm, const int32_t* ctx_lens) {
   if (!ctx_lens) return LUKV_ERR_INVALID_ARG;
-  if (dm->S > kMaxRaggedSeqs) return LUKV_ERR_UNSUPPORTED;
+  if (dm->S > kMaxRaggedSeqs || dm->keydiff) return LUKV_ERR_UNSUPPORTED;
   for (int q = 0; q < dm->S; ++q) {
     const int Tq = ctx_lens[q];
     if (Tq <= dm->w || Tq > dm->T || dm->n_sink > Tq - dm->w) return LUKV_ERR_INVALID_ARG;
@@ -57,7 +57,8 @@ static int attach_seq_lens(Dims* dm, const int32_t* ctx_lens) {
 // Validates the parameter block and fills Dims.
 static int make_dims(const lukv_params_t* p, Dims* dm) {
   if (!p) return LUKV_ERR_INVALID_ARG;
-  if (p->flags != 0) return LUKV_ERR_INVALID_ARG;
+  if ((p->flags & ~LUKV_FLAG_KEYDIFF) != 0) return LUKV_ERR_INVALID_ARG;
+  if ((p->flags & LUKV_FLAG_KEYDIFF) && p->pool_kernel != 1) return LUKV_ERR_INVALID_ARG;
   if (p->batch < 1 || p->n_layers < 1 || p->n_kv_heads < 1 || p->gqa_group < 1 || p->ctx_len < 2 || p->window < 1 ||
       p->window >= p->ctx_len || p->pool_kernel < 1 || p->curve_points < 2)
     return LUKV_ERR_INVALID_ARG;
@@ -89,6 +90,7 @@ static int make_dims(const lukv_params_t* p, Dims* dm) {
   dm->n_sink = p->n_sink;
   dm->min_keep = p->min_keep;
   dm->seq_T = nullptr;
+  dm->keydiff = (p->flags & LUKV_FLAG_KEYDIFF) != 0;
   const double fl = ceil((double)p->min_keep * (double)dm->n);
   dm->floor_tok = fl < 0.0 ? 0 : (fl > (double)dm->n ? dm->n : (int)fl);
   return LUKV_OK;
@@ -125,6 +127,7 @@ static HeadRange all_heads(const Dims& dm) { return HeadRange{0, (int)dm.heads()
 
 static cudaError_t run_score(const Dims& dm, const void* q, const void* k, const Workspace& ws, float* pooled_out,
                              int32_t* dev_status, LaunchCtx& lc) {
+  if (dm.keydiff) return launch_keydiff(dm, k, pooled_out, ws.stats, dev_status, 0, lc);  // nothing to pool
   cudaError_t e = (score_tc_supported(dm) && !force_simt())
                       ? launch_score_tc(dm, q, k, ws, dev_status, all_heads(dm), true, 0, lc)
                       : launch_score_simt(dm, q, k, ws, lc);
@@ -169,7 +172,8 @@ static int run_compress(const Dims& dm, const void* q_win, const void* k, const 
                         bool overlap) {
   if (dev_status && cudaMemsetAsync(dev_status, 0, sizeof(int32_t), lc.st) != cudaSuccess) return LUKV_ERR_CUDA;
   const bool tc = score_tc_supported(dm) && !force_simt();
-  SideStream* side = (overlap && tc) ? side_stream() : nullptr;
+  // the persistent scorers (tensor-core, KeyDiff) leave one SM to the allocation kernels of the auxiliary stream
+  SideStream* side = (overlap && (tc || dm.keydiff)) ? side_stream() : nullptr;
   int rc = LUKV_OK;
   if (side) {
     std::lock_guard<std::mutex> in_use(side->use);
@@ -180,9 +184,12 @@ static int run_compress(const Dims& dm, const void* q_win, const void* k, const 
     if (launch_allocate(dm, curves, budgets_in, w.gains, budgets, offsets, ls) != cudaSuccess) rc = LUKV_ERR_CUDA;
     if (cudaEventRecord(side->join, ls.st) != cudaSuccess) rc = LUKV_ERR_CUDA;
     lc.launches += ls.launches;
-    if (rc == LUKV_OK && (launch_score_tc(dm, q_win, k, w, dev_status, all_heads(dm), true, 1, lc) != cudaSuccess ||
-                          launch_pool(dm, w.raw, w.pooled, all_heads(dm), lc) != cudaSuccess))
+    if (rc == LUKV_OK && dm.keydiff) {
+      if (launch_keydiff(dm, k, w.pooled, w.stats, dev_status, 1, lc) != cudaSuccess) rc = LUKV_ERR_CUDA;
+    } else if (rc == LUKV_OK && (launch_score_tc(dm, q_win, k, w, dev_status, all_heads(dm), true, 1, lc) != cudaSuccess ||
+                                 launch_pool(dm, w.raw, w.pooled, all_heads(dm), lc) != cudaSuccess)) {
       rc = LUKV_ERR_CUDA;
+    }
     // join even after a failure: the caller's stream must not run ahead of work already enqueued
     if (cudaStreamWaitEvent(lc.st, side->join, 0) != cudaSuccess) rc = LUKV_ERR_CUDA;
     if (rc != LUKV_OK) return rc;
@@ -205,9 +212,10 @@ static int check_compress_args(const lukv_params_t* params, const void* q_win, c
   int rc = make_dims(params, dm);
   if (rc != LUKV_OK) return rc;
   if (ragged && (rc = attach_seq_lens(dm, ctx_lens)) != LUKV_OK) return rc;
-  if (!q_win || !k || !v || !curves || !budgets_in || !k_out || !v_out || !kept_idx || !budgets || !offsets ||
-      !aligned16(q_win) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
+  if (!k || !v || !curves || !budgets_in || !k_out || !v_out || !kept_idx || !budgets || !offsets ||
+      !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
     return LUKV_ERR_INVALID_ARG;
+  if (!dm->keydiff && (!q_win || !aligned16(q_win))) return LUKV_ERR_INVALID_ARG;
   int64_t rows;
   if ((rc = check_budgets(*dm, budgets_in, &rows)) != LUKV_OK) return rc;
   if (rows >= (int64_t)1 << 31) return LUKV_ERR_UNSUPPORTED;
@@ -235,7 +243,7 @@ int lukv_score(const lukv_params_t* params, const void* q_win, const void* k, fl
   Dims dm;
   int rc = make_dims(params, &dm);
   if (rc != LUKV_OK) return rc;
-  if (!q_win || !k || !scores || !aligned16(q_win) || !aligned16(k)) return LUKV_ERR_INVALID_ARG;
+  if (!k || !scores || !aligned16(k) || (!dm.keydiff && (!q_win || !aligned16(q_win)))) return LUKV_ERR_INVALID_ARG;
   Workspace w;
   if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
   LaunchCtx lc;
@@ -256,7 +264,7 @@ int lukv_score_keydiff(const lukv_params_t* params, const void* k, float* scores
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;
   if (dev_status && cudaMemsetAsync(dev_status, 0, sizeof(int32_t), lc.st) != cudaSuccess) return LUKV_ERR_CUDA;
-  if (launch_keydiff(dm, k, scores, w.stats, dev_status, lc) != cudaSuccess) return LUKV_ERR_CUDA;
+  if (launch_keydiff(dm, k, scores, w.stats, dev_status, 0, lc) != cudaSuccess) return LUKV_ERR_CUDA;
   g_last_launches = lc.launches;
   return LUKV_OK;
 }
@@ -267,7 +275,7 @@ int lukv_score_ragged(const lukv_params_t* params, const int32_t* ctx_lens, cons
   int rc = make_dims(params, &dm);
   if (rc != LUKV_OK) return rc;
   if ((rc = attach_seq_lens(&dm, ctx_lens)) != LUKV_OK) return rc;
-  if (!q_win || !k || !scores || !aligned16(q_win) || !aligned16(k)) return LUKV_ERR_INVALID_ARG;
+  if (!k || !scores || !aligned16(k) || (!dm.keydiff && (!q_win || !aligned16(q_win)))) return LUKV_ERR_INVALID_ARG;
   Workspace w;
   if ((rc = check_ws(dm, ws, ws_bytes, &w)) != LUKV_OK) return rc;
   LaunchCtx lc;

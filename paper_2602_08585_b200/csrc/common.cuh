@@ -26,6 +26,7 @@ struct Dims {
   // T, n and the tensor strides then describe the longest one.  nullptr: every sequence has length T.
   const int32_t* seq_T = nullptr;
   float min_keep = 0.f;  // as given (the per-sequence floors of a ragged call are derived from it)
+  bool keydiff = false;  // stage (a) is the KeyDiff metric (keys only, no pooling)
   int64_t heads() const { return (int64_t)S * N; }
   size_t esize() const { return dtype == LUKV_DTYPE_BF16 ? 2 : 4; }
 };
@@ -132,7 +133,7 @@ cudaError_t launch_build_curves(const Dims& dm, const float* scores, const float
 // KeyDiff proxy scores (key-only metric): scores [heads][n]; scratch of keydiff_scratch_bytes().
 size_t keydiff_scratch_bytes(const Dims& dm);
 cudaError_t launch_keydiff(const Dims& dm, const void* k, float* scores, float* scratch, int32_t* dev_status,
-                           LaunchCtx& lc);
+                           int spare_sms, LaunchCtx& lc);
 // Oracle importance of Sec. 4.1 from decode queries, the cache and the output projection.
 size_t importance_workspace_bytes(const Dims& dm, int k_max);
 cudaError_t launch_importance(const Dims& dm, int k_max, int d_model, const void* q_dec, const void* k, const void* v,

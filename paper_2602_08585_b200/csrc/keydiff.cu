@@ -364,7 +364,7 @@ size_t kd_head_bytes(const Dims& dm) { return kd_align((size_t)dm.heads() * size
 
 template <typename TIn, int D>
 cudaError_t launch_keydiff_t(const Dims& dm, const void* k, float* scores, float* scratch, int32_t* dev_status,
-                             LaunchCtx& lc) {
+                             int spare_sms, LaunchCtx& lc) {
   auto kern = keydiff_kernel<TIn, D>;
   int dev = 0, sms = 0, per_sm = 0;
   cudaError_t e;
@@ -375,6 +375,7 @@ cudaError_t launch_keydiff_t(const Dims& dm, const void* k, float* scores, float
   if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kKdThreads, kKdRingBytes)) != cudaSuccess)
     return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+  if (spare_sms > 0 && sms > 8 * spare_sms) sms -= spare_sms;  // kernels of another stream keep these
   KdArgs a;
   unsigned char* sc = reinterpret_cast<unsigned char*>(scratch);
   a.k = static_cast<const unsigned char*>(k);
@@ -407,12 +408,12 @@ size_t keydiff_scratch_bytes(const Dims& dm) {
 }
 
 cudaError_t launch_keydiff(const Dims& dm, const void* k, float* scores, float* scratch, int32_t* dev_status,
-                           LaunchCtx& lc) {
+                           int spare_sms, LaunchCtx& lc) {
   if (dm.dtype == LUKV_DTYPE_BF16)
-    return dm.d == 128 ? launch_keydiff_t<__nv_bfloat16, 128>(dm, k, scores, scratch, dev_status, lc)
-                       : launch_keydiff_t<__nv_bfloat16, 64>(dm, k, scores, scratch, dev_status, lc);
-  return dm.d == 128 ? launch_keydiff_t<float, 128>(dm, k, scores, scratch, dev_status, lc)
-                     : launch_keydiff_t<float, 64>(dm, k, scores, scratch, dev_status, lc);
+    return dm.d == 128 ? launch_keydiff_t<__nv_bfloat16, 128>(dm, k, scores, scratch, dev_status, spare_sms, lc)
+                       : launch_keydiff_t<__nv_bfloat16, 64>(dm, k, scores, scratch, dev_status, spare_sms, lc);
+  return dm.d == 128 ? launch_keydiff_t<float, 128>(dm, k, scores, scratch, dev_status, spare_sms, lc)
+                     : launch_keydiff_t<float, 64>(dm, k, scores, scratch, dev_status, spare_sms, lc);
 }
 
 }  // namespace lukv

@@ -19,6 +19,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BUDGET, ERR_WORKSPACE_TOO_SMALL = -1, -2, -3, -4
 ERR_OUTPUT_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
 DTYPE_BF16, DTYPE_FP32 = 0, 1
+FLAG_KEYDIFF = 1  # params.flags: stage (a) is the KeyDiff metric
 
 EXPORTS = ("lukv_workspace_bytes", "lukv_score", "lukv_allocate", "lukv_select_gather", "lukv_compress",
            "lukv_strerror", "lukv_last_launch_count", "lukv_compress_profile", "lukv_allocate_static",
@@ -101,12 +102,12 @@ def strerror(code: int) -> str:
 
 
 def make_params(S: int, L: int, H: int, G: int, d: int, T: int, w: int, kp: int, dtype, P: int,
-                scale: float = 0.0, n_sink: int = 0, min_keep: float = 0.0) -> Params:
+                scale: float = 0.0, n_sink: int = 0, min_keep: float = 0.0, flags: int = 0) -> Params:
     if isinstance(dtype, torch.dtype):
         dtype = {torch.bfloat16: DTYPE_BF16, torch.float32: DTYPE_FP32}[dtype]
     elif isinstance(dtype, str):
         dtype = {"bf16": DTYPE_BF16, "fp32": DTYPE_FP32}[dtype]
-    return Params(S, L, H, G, d, T, w, kp, int(dtype), P, float(scale), 0, int(n_sink), float(min_keep))
+    return Params(S, L, H, G, d, T, w, kp, int(dtype), P, float(scale), int(flags), int(n_sink), float(min_keep))
 
 
 def _ptr(t) -> Optional[int]:

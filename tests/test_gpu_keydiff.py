@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 import torch
 
-from paper_2602_08585_b200 import lukv
+from paper_2602_08585_b200 import lukv, synth
 from gpu_helpers import bits, gpu_select_gather
 
 pytestmark = pytest.mark.gpu
@@ -128,3 +128,75 @@ def test_keydiff_selection_and_gather(oracle):
             assert np.all(np.abs(ref_scores.reshape(N, n)[u][diff] - t) <= 2 * ATOL)
         assert kept2[o + b] == n                      # the recent window of one position
     assert same / total >= 0.999
+
+
+def _kept_close(kept_gpu, kept_ref, budgets, offsets, ref_scores, w):
+    """Same kept sets, up to positions whose oracle scores lie within the tolerance of the head's threshold."""
+    n = ref_scores.shape[-1]
+    flat = ref_scores.reshape(-1, n)
+    same = total = 0
+    for u, b in enumerate(budgets.reshape(-1)):
+        o = offsets[u]
+        assert np.array_equal(kept_gpu[o + b:o + b + w], np.arange(n, n + w))      # the recent window
+        if b == 0:
+            continue
+        a, r = kept_gpu[o:o + b], kept_ref[o:o + b]
+        assert np.all(np.diff(a) > 0)
+        same += len(np.intersect1d(a, r))
+        total += b
+        diff = np.setxor1d(a, r)
+        if len(diff):
+            t = np.sort(flat[u])[::-1][b - 1]
+            assert np.all(np.abs(flat[u][diff] - t) <= 2 * ATOL)
+    return same / max(total, 1)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_keydiff_whole_path_by_flag(oracle, dtype):
+    """lukv_compress with LUKV_FLAG_KEYDIFF: KeyDiff scores -> joint allocation from the curves -> per-head top-b ->
+    gather, against the same chain of oracle functions.  No queries are passed."""
+    wl = synth.scaled(synth.CONFIGS["llama8b_1layer_8k"], S=2, L=2, H=3, T=4096, w=1, kp=1, P=129, dtype=dtype,
+                      d=128 if dtype == "bf16" else 64)
+    _, k, v = synth.gen_tensors(wl, "cpu")
+    curves = synth.gen_curves(wl)
+    n = wl.T - wl.w
+    Bs = [int(0.2 * wl.N * n), int(0.55 * wl.N * n)]
+    p = lukv.make_params(wl.S, wl.L, wl.H, wl.G, wl.d, wl.T, wl.w, wl.kp, wl.dtype, wl.P, flags=lukv.FLAG_KEYDIFF)
+    ws = lukv.alloc_workspace(p)
+    out = lukv.Outputs(p, Bs)
+    kc, vc = k.cuda(), v.cuda()
+    lukv.lukv_compress(p, None, kc, vc, torch.from_numpy(curves).cuda(), Bs, out.k_out, out.v_out, out.kept_idx,
+                       out.budgets, out.offsets, out.rows, out.dev_status, ws)
+    torch.cuda.synchronize()
+    assert int(out.dev_status.item()) == 0
+    ref_scores = oracle.keydiff(bits(k), wl.w)
+    rb, ro = oracle.allocate(curves, wl.T, wl.w, Bs)
+    np.testing.assert_array_equal(out.budgets.cpu().numpy(), rb)
+    np.testing.assert_array_equal(out.offsets.cpu().numpy(), ro)
+    U = wl.S * wl.N
+    rk, rv, rkept = oracle.select_gather(ref_scores.reshape(U, n), rb, ro, bits(k).reshape(U, wl.T, wl.d),
+                                         bits(v).reshape(U, wl.T, wl.d), wl.w)
+    kept = out.kept_idx.cpu().numpy()
+    assert _kept_close(kept, rkept, rb, ro, ref_scores, wl.w) >= 0.999
+    # the gathered rows are the rows the kept indices name, bit for bit
+    kb, vb = bits(k).reshape(U, wl.T, wl.d), bits(v).reshape(U, wl.T, wl.d)
+    head_of_row = np.repeat(np.arange(U), np.diff(ro))
+    np.testing.assert_array_equal(bits(out.k_out), kb[head_of_row, kept])
+    np.testing.assert_array_equal(bits(out.v_out), vb[head_of_row, kept])
+    # lukv_score with the flag returns the KeyDiff scores
+    scores = torch.empty((wl.S, wl.N, n), dtype=torch.float32, device="cuda")
+    lukv.lukv_score(p, None, kc, scores, ws)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(scores.cpu().numpy(), ref_scores, rtol=0, atol=ATOL)
+
+
+def test_keydiff_flag_argument_errors():
+    f = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    pooled = lukv.make_params(1, 1, 2, 1, 64, 256, 1, 7, "bf16", 2, flags=lukv.FLAG_KEYDIFF)   # the metric is not pooled
+    assert lukv.lukv_score(pooled, None, f, f, f, check=False) == lukv.ERR_INVALID_ARG
+    unknown = lukv.make_params(1, 1, 2, 1, 64, 256, 1, 1, "bf16", 2, flags=2)
+    assert lukv.lukv_score(unknown, None, f, f, f, check=False) == lukv.ERR_INVALID_ARG
+    plain = lukv.make_params(1, 1, 2, 1, 64, 256, 1, 1, "bf16", 2)
+    assert lukv.lukv_score(plain, None, f, f, f, check=False) == lukv.ERR_INVALID_ARG           # queries are required
+    flagged = lukv.make_params(2, 1, 2, 1, 64, 256, 1, 1, "bf16", 2, flags=lukv.FLAG_KEYDIFF)
+    assert lukv.lukv_score_ragged(flagged, [256, 128], None, f, f, f, check=False) == lukv.ERR_UNSUPPORTED
