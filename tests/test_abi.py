@@ -99,7 +99,9 @@ def test_argument_errors_come_back_before_any_launch():
     assert lukv.lukv_compress(p, f, f, f, f, [n_max + 5], f, f, f, f, f, 1 << 30, None, f,
                               check=False) == lukv.ERR_BUDGET
     bad = lukv.make_params(1, 2, 2, 2, 64, 256, 8, 3, "bf16", 17)
-    bad.flags = 1
+    bad.flags = 2                                     # an unknown flag bit
+    assert lukv.lukv_score(bad, f, f, f, f, check=False) == lukv.ERR_INVALID_ARG
+    bad.flags = lukv.FLAG_KEYDIFF                     # the KeyDiff metric is not pooled: pool_kernel must be 1
     assert lukv.lukv_score(bad, f, f, f, f, check=False) == lukv.ERR_INVALID_ARG
 
 
