@@ -1,15 +1,21 @@
 // Stages (c) and (d): per-head variable-k top-k selection and the packed gather.
-//   select_kernel  one CTA per head: the b-th largest score is found digit by digit (11, 11
+//   select_kernel  one CTA per head, or a thread-block cluster of 2, 4 or 8 CTAs per head that merge their
+//                  histograms and counts through distributed shared memory (long contexts; few heads):
+//                  the b-th largest score is found digit by digit (11, 11
 //                  and 10 bits) over the order-preserving integer image of the scores, each
 //                  digit from a shared-memory histogram, then the kept positions are emitted in
 //                  ascending order: everything above the threshold plus the first
 //                  (lowest-position) ties.  This realises M^pi(b) of Sec. 3.2 / the
 //                  "Eviction" step of Sec. 4.3 without a full sort.
 //   gather_kernel  copies the kept K/V rows into the packed cache, 16 bytes per lane.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace lukv {
 namespace {
+
+namespace cg = cooperative_groups;
 
 constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
@@ -26,12 +32,13 @@ __device__ __forceinline__ uint32_t key_at(const float* src, int j, int n_sink) 
   return j < n_sink ? 0xFFFFFFFFu : score_key(src[j]);
 }
 
-// One CTA per head.  Warp wv owns the positions [wv*span, (wv+1)*span) and lane l of it the
-// positions wv*span + e*32 + l, so loads are coalesced and position order is (warp, e, lane).
+// One CTA per head (CLUSTER false) or one cluster of CTAs per head (CLUSTER true; CTA r of the cluster owns the
+// positions [r*32*span, (r+1)*32*span)).  Warp wv of a CTA owns span consecutive positions and lane l of it the
+// positions e*32 + l of those, so loads are coalesced and position order is (CTA, warp, e, lane).
 // EPT > 0: span = 32*EPT and the thread keeps its EPT keys in registers (n <= 1024*EPT).
 // EPT == 0: span is a multiple of 32 given by the host and the keys are re-read from memory
 // in every round (long contexts).
-template <int EPT>
+template <int EPT, bool CLUSTER>
 __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __restrict__ pooled,
                                                                 const int32_t* __restrict__ budgets,
                                                                 const int32_t* __restrict__ offsets,
@@ -41,7 +48,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
   __shared__ int hist[2048];
   __shared__ int scan_gt[kSelWarps], scan_eq[kSelWarps];
   __shared__ int sel_digit, sel_want;
-  const int u = head0 + blockIdx.x, tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
+  __shared__ int cta_tot[2];  // keys of this CTA above / equal to the threshold
+  static_assert(!CLUSTER || EPT > 0, "a cluster keeps its keys in registers");
+  cg::cluster_group cluster = cg::this_cluster();
+  const int csize = CLUSTER ? (int)cluster.num_blocks() : 1, crank = CLUSTER ? (int)cluster.block_rank() : 0;
+  const int u = head0 + (int)blockIdx.x / csize, tid = threadIdx.x, lane = tid & 31, wv = tid >> 5;
   const int b = budgets[u];
   const long long off = offsets[u];
   // n_stride: row stride of the scores (the longest sequence); n: rankable positions of this head's sequence
@@ -51,12 +62,13 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
   const long long room = rows_cap - off;  // rows of this head that fit in the output
 
   // window rows follow the selected ones
-  for (int t = tid; t < w; t += kSelThreads)
-    if (b + t < room) out[b + t] = n + t;
-  if (b <= 0) return;
+  if (crank == 0)
+    for (int t = tid; t < w; t += kSelThreads)
+      if (b + t < room) out[b + t] = n + t;
+  if (b <= 0) return;  // the whole cluster leaves
 
   const int span = EPT > 0 ? 32 * EPT : span_rt;
-  const int base = wv * span + lane;
+  const int base = (crank * kSelWarps + wv) * span + lane;
   const int iters = span >> 5;
   uint32_t keys[EPT > 0 ? EPT : 1];
   if (EPT > 0) {
@@ -65,7 +77,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
       const int j = base + 32 * e;
       keys[e] = j < n ? score_key(src[j]) : 0u;
     }
-    if (wv * span < n_sink) {  // only the warps whose span starts below n_sink hold sink positions
+    if (base - lane < n_sink) {  // only the warps whose span starts below n_sink hold sink positions
 #pragma unroll
       for (int e = 0; e < EPT; ++e)
         if (base + 32 * e < n_sink) keys[e] = 0xFFFFFFFFu;
@@ -99,11 +111,22 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
           count(j < n ? key_at(src, j, n_sink) : 0u, j);
         }
       }
-      __syncthreads();
+      if (CLUSTER) cluster.sync(); else __syncthreads();  // every histogram of the head is complete
       // thread t owns the bins [t*per, t*per+per); suffix sums over the threads, from the top
       const int per = bins / kSelThreads;  // 2 or 1
-      int mine = 0;
-      for (int i = 0; i < per; ++i) mine += hist[tid * per + i];
+      // the bins of this thread, added over the CTAs of the head (every CTA computes the same)
+      int merged0 = 0, merged1 = 0;
+      if (CLUSTER) {
+        for (int c = 0; c < csize; ++c) {
+          const int* remote = cluster.map_shared_rank(hist, c) + tid * per;
+          merged0 += remote[0];
+          if (per == 2) merged1 += remote[1];
+        }
+      } else {
+        merged0 = hist[tid * per];
+        if (per == 2) merged1 = hist[tid * per + 1];
+      }
+      const int mine = merged0 + merged1;
       int incl = mine;  // sum over the lanes >= this one
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
@@ -118,7 +141,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
       if (higher < want && want <= higher + mine) {  // exactly one thread: the digit is in its bins
         int run = higher;
         for (int i = per - 1; i >= 0; --i) {
-          const int c = hist[tid * per + i];
+          const int c = i ? merged1 : merged0;
           if (want <= run + c) {
             sel_digit = tid * per + i;
             sel_want = want - run;
@@ -127,7 +150,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
           run += c;
         }
       }
-      __syncthreads();
+      if (CLUSTER) cluster.sync(); else __syncthreads();  // the histograms may be cleared again
       thr |= (uint32_t)sel_digit << shift;
       want = sel_want;
     }
@@ -163,6 +186,27 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const float* __r
       run_eq += scan_eq[x];
     }
     total_gt += scan_gt[x];
+  }
+  if (CLUSTER) {
+    // the CTAs before this one along the positions come first; the totals run over the whole head
+    if (tid == 0) {
+      int eq = 0;
+      for (int x = 0; x < kSelWarps; ++x) eq += scan_eq[x];
+      cta_tot[0] = total_gt;
+      cta_tot[1] = eq;
+    }
+    cluster.sync();
+    total_gt = 0;
+    for (int c = 0; c < csize; ++c) {
+      const int* tot = cluster.map_shared_rank(cta_tot, c);
+      const int g = tot[0], q = tot[1];
+      if (c < crank) {
+        run_gt += g;
+        run_eq += q;
+      }
+      total_gt += g;
+    }
+    cluster.sync();  // no CTA of the cluster exits while another may still read its shared memory
   }
   const int k_eq = b - total_gt;  // ties to keep (>= 1)
 
@@ -281,20 +325,42 @@ cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* bu
   const int hps = dm.seq_T ? dm.N : 0;
   if (dm.seq_T)
     for (int q = 0; q < dm.S; ++q) sl.T[q] = dm.seq_T[q];
-  if (n <= kSelThreads * 2)
-    select_kernel<2><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
-                                                    dm.n_sink, sl, hps);
-  else if (n <= kSelThreads * 8)
-    select_kernel<8><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
-                                                    dm.n_sink, sl, hps);
-  else if (n <= kSelThreads * 32)
-    select_kernel<32><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0,
-                                                    dm.n_sink, sl, hps);
-  else {
+  // Keys per thread (in registers) and CTAs per head.  Up to 32768 positions: one CTA with 2, 8 or 32 keys per
+  // thread (a cluster's barriers cost more than they save there).  Up to 262144: the smallest cluster (2, 4 or 8
+  // CTAs) that covers the head with 32 keys per thread; small clusters are placed and synchronised faster than large
+  // ones.  Beyond: one CTA that re-reads its keys from memory in every round.
+  int ept = 0, csize = 1;
+  if (n <= kSelThreads * 32) {
+    ept = n <= kSelThreads * 2 ? 2 : n <= kSelThreads * 8 ? 8 : 32;
+  } else {
+    for (int c : {2, 4, 8})
+      if (!ept && (long long)c * kSelThreads * 32 >= n) ept = 32, csize = c;
+  }
+  if (ept == 0) {
     const int per_warp = (n + kSelWarps - 1) / kSelWarps;
     const int span = (per_warp + 31) & ~31;
-    select_kernel<0><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, span, hr.h0,
-                                                   dm.n_sink, sl, hps);
+    select_kernel<0, false><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, span,
+                                                          hr.h0, dm.n_sink, sl, hps);
+  } else if (csize == 1) {
+    auto kern = ept == 2 ? select_kernel<2, false> : ept == 8 ? select_kernel<8, false> : select_kernel<32, false>;
+    kern<<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0, dm.n_sink, sl,
+                                       hps);
+  } else {
+    auto kern = select_kernel<32, true>;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid * csize);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = csize;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, scores, budgets, offsets, kept_idx, (long long)rows_cap, n,
+                                             dm.w, 0, hr.h0, dm.n_sink, sl, hps);
+    if (e != cudaSuccess) return e;
   }
   lc.mark("select");
   return cudaGetLastError();

@@ -183,6 +183,35 @@ def test_select_gather_long_context_single_head(oracle):
     _select_case(oracle, 1, 1, T, w, d, torch.bfloat16, [90000], scores)
 
 
+@pytest.mark.parametrize("T,n_sink", [(70000, 0), (131072 + 64, 4), (200000, 0), (262144 + 32, 0), (270000, 4)])
+def test_select_gather_cluster_and_streaming_paths(oracle, T, n_sink):
+    """Contexts beyond 32768 positions: clusters of 4 and 8 CTAs per head that merge their histograms (clusters of 2:
+    the 33000 and 40000 cases above), and beyond 262144 positions one CTA that re-reads its keys.  Plateaus put ties
+    on the cut; one head keeps nothing, one nearly everything."""
+    w, d, S, N = 32, 64, 1, 3
+    n = T - w
+    rng = np.random.default_rng(T)
+    scores = rng.random((S, N, n)).astype(np.float32) ** 8
+    scores[0, 1] = np.repeat(rng.random(n // 5 + 1).astype(np.float32), 5)[:n]
+    budgets = np.asarray([[n // 3, n - 7, 0]], np.int32)
+    if n_sink:
+        scores[0, 0, :n_sink] = 0.0                    # sinks rank first whatever their scores
+    g = torch.Generator().manual_seed(T)
+    k = torch.randn((S, 1, N, T, d), generator=g).to(torch.bfloat16)
+    v = torch.randn((S, 1, N, T, d), generator=g).to(torch.bfloat16)
+    offsets = np.concatenate([[0], np.cumsum(budgets.reshape(-1) + w)]).astype(np.int32)
+    rows = int(offsets[-1])
+    p = lukv.make_params(S, 1, N, 1, d, T, w, 1, torch.bfloat16, 2, n_sink=n_sink)
+    k_out, v_out, kept = gpu_select_gather(p, torch.from_numpy(scores).cuda(), torch.from_numpy(budgets).cuda(),
+                                           torch.from_numpy(offsets).cuda(), k.cuda(), v.cuda(), rows, pad_rows=3)
+    rk, rv, rkept = oracle.select_gather(scores.reshape(N, n), budgets, offsets, bits(k).reshape(N, T, d),
+                                         bits(v).reshape(N, T, d), w, n_sink=n_sink)
+    np.testing.assert_array_equal(kept.cpu().numpy()[:rows], rkept)
+    np.testing.assert_array_equal(bits(k_out)[:rows], rk)
+    np.testing.assert_array_equal(bits(v_out)[:rows], rv)
+    assert torch.all(kept[rows:] == -1)
+
+
 # ---- the whole path ------------------------------------------------------------------------------
 
 def _compress_case(oracle, wl, min_agreement=0.999):
