@@ -134,6 +134,10 @@ cudaError_t launch_build_curves(const Dims& dm, const float* scores, const float
 size_t keydiff_scratch_bytes(const Dims& dm);
 cudaError_t launch_keydiff(const Dims& dm, const void* k, float* scores, float* scratch, int32_t* dev_status,
                            int spare_sms, LaunchCtx& lc);
+// Value norms || v_j W_O^(g) ||_2 of the oracle importance on the tensor cores (bf16, d = 128): vnorm [heads][G][n].
+bool value_norm_tc_supported(const Dims& dm);
+cudaError_t launch_value_norm_tc(const Dims& dm, int d_model, const void* v, const void* w_o, float* vnorm,
+                                 LaunchCtx& lc);
 // Oracle importance of Sec. 4.1 from decode queries, the cache and the output projection.
 size_t importance_workspace_bytes(const Dims& dm, int k_max);
 cudaError_t launch_importance(const Dims& dm, int k_max, int d_model, const void* q_dec, const void* k, const void* v,

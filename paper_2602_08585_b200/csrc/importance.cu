@@ -8,6 +8,8 @@
 //   imp_lse_kernel      row log-sum-exp of every (head, g, step), exp2 domain
 //   imp_kernel          probabilities x value norms, summed over g inside a thread, maximum over the steps
 //   imp_normalize_kernel  one CTA per (sequence, layer): fp64 total in a fixed order, then the division
+#include <cstdlib>
+
 #include "simt_tile.cuh"
 
 namespace lukv {
@@ -244,6 +246,12 @@ __global__ void __launch_bounds__(1024) imp_normalize_kernel(float* __restrict__
   for (long long i = threadIdx.x; i < count; i += blockDim.x) base[i] = (float)((double)base[i] / total);
 }
 
+// LUKV_FORCE_SIMT=1 keeps the value norms on the FP32 pipes (for A/B checks; read at every call).
+bool value_norm_force_simt() {
+  const char* e = getenv("LUKV_FORCE_SIMT");
+  return e && e[0] == '1';
+}
+
 template <typename TIn, int D>
 cudaError_t launch_importance_t(const Dims& dm, ImpDims id, const void* q_dec, const void* k, const void* v,
                                 const void* k_dec, const void* w_o, bool normalize, float* importance, float* vnorm,
@@ -258,8 +266,12 @@ cudaError_t launch_importance_t(const Dims& dm, ImpDims id, const void* q_dec, c
   if ((e = cudaFuncSetAttribute(ki, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   const unsigned heads = (unsigned)dm.heads();
   const unsigned pos_tiles = (unsigned)((dm.n + kTile - 1) / kTile);
-  kn<<<dim3(heads * id.G, pos_tiles), kSimtThreads, smem, lc.st>>>((const TIn*)v, (const TIn*)w_o, vnorm, id);
-  lc.mark("value_norm");
+  if (value_norm_tc_supported(dm) && !value_norm_force_simt()) {
+    if ((e = launch_value_norm_tc(dm, id.Dm, v, w_o, vnorm, lc)) != cudaSuccess) return e;
+  } else {
+    kn<<<dim3(heads * id.G, pos_tiles), kSimtThreads, smem, lc.st>>>((const TIn*)v, (const TIn*)w_o, vnorm, id);
+    lc.mark("value_norm");
+  }
   kl<<<dim3(heads, (unsigned)((id.Kmax + 15) / 16)), kSimtThreads, smem, lc.st>>>((const TIn*)q_dec, (const TIn*)k,
                                                                                  (const TIn*)k_dec, lse, id);
   lc.mark("imp_lse");

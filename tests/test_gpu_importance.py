@@ -44,6 +44,10 @@ SHAPES = [
     (1, 1, 1, 7, 128, 600, 32, 33, 64, torch.bfloat16, True, False),        # GQA group 7: two chunks of query heads
     (1, 2, 3, 2, 64, 1025, 7, 16, 130, torch.bfloat16, False, True),        # no decode keys
     (1, 1, 2, 4, 128, 4000, 32, 8, 256, torch.bfloat16, True, True),        # the paper's calibration length
+    # value norms on the tensor cores (bf16, d = 128): projection panels of 256 columns, chunks of 4096 positions
+    (1, 2, 1, 2, 128, 700, 32, 4, 516, torch.bfloat16, False, True),        # three panels, the last one ragged
+    (1, 1, 2, 1, 128, 300, 8, 3, 77, torch.bfloat16, True, False),          # odd width: the unvectorised panel writer
+    (2, 1, 1, 2, 128, 4096 + 700, 32, 2, 264, torch.bfloat16, False, True), # two position chunks per head
 ]
 
 
@@ -58,6 +62,18 @@ def test_importance_matches_oracle(oracle, shape):
     _close(got, ref)
     if normalize:
         np.testing.assert_allclose(got.reshape(S, L, -1).sum(axis=2), 1.0, rtol=1e-4)
+
+
+def test_value_norms_tensor_core_against_fp32_pipes(monkeypatch):
+    """The two value-norm kernels (tensor cores; FP32 pipes, kept for other shapes) agree far inside the tolerance:
+    bf16 products are exact in fp32 and both accumulate in fp32."""
+    S, L, H, G, d, T, w, Kmax, Dm = 1, 2, 2, 4, 128, 2000, 32, 4, 1024
+    q, k, v, kd, wo = _inputs(S, L, H, G, d, T, Kmax, Dm, torch.bfloat16, seed=21)
+    p = lukv.make_params(S, L, H, G, d, T, w, 1, torch.bfloat16, 2)
+    tc = gpu_importance(p, Kmax, Dm, q, k, v, kd, wo, False)
+    monkeypatch.setenv("LUKV_FORCE_SIMT", "1")
+    simt = gpu_importance(p, Kmax, Dm, q, k, v, kd, wo, False)
+    np.testing.assert_allclose(tc, simt, rtol=2e-5, atol=1e-30)
 
 
 def test_importance_argument_errors():
