@@ -204,6 +204,15 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def bf16_peak_tflops():
+    """Measured dense bf16 rate of a kernel timed alone (burst), else the earlier measurement on this machine."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops"])
+    except Exception:
+        return 1590.0
+
+
 def kernel_bytes(name, wl, rows):
     """Algorithmic bytes one launch of a kernel must move (inputs read once + outputs written once)."""
     es = 2 if wl.dtype == "bf16" else 4
@@ -624,7 +633,8 @@ def run_profile_path(args):
                            "relaxation_gap": (exact_val - greedy_raw) / exact_val},
         "oracle_importance": {"ms_per_call": imp_ms, "queries": 1, "heads": wl.N, "gqa_group": wl.G,
                               "positions": Tc - wl.w, "decode_steps": Kd, "d_model": Dm, "launches": imp_launches,
-                              "flops": imp_flops, "tflops": imp_flops / (imp_ms * 1e-3) / 1e12},
+                              "flops": imp_flops, "tflops": imp_flops / (imp_ms * 1e-3) / 1e12,
+                              "frac_of_measured_bf16_peak": imp_flops / (imp_ms * 1e-3) / 1e12 / bf16_peak_tflops()},
         "keydiff_scores": {"ms_per_call": keydiff_ms, "launches": keydiff_launches,
                            "algorithmic_bytes": keydiff_bytes, "gbs": keydiff_bytes / (keydiff_ms * 1e-3) / 1e9,
                            "frac_of_measured_hbm_peak": keydiff_bytes / (keydiff_ms * 1e-3) / 1e9 / measured_peak()[0],
