@@ -118,6 +118,9 @@ LUKV_API int lukv_workspace_bytes(const lukv_params_t* params, size_t* bytes /* 
  *                             belongs to KV head h)
  *   k      [S][L][H][T][d]
  *   scores [S][N][n] fp32     out: pooled scores (>= 0)
+ * This call has no device status word: should a bounded wait of the scorer run out (see dev_status of
+ * lukv_compress; it needs the device to be taken away in mid-kernel), the scores are undefined and nothing
+ * reports it.  lukv_compress and lukv_score_keydiff report it.
  */
 LUKV_API int lukv_score(const lukv_params_t* params, const void* q_win, const void* k, float* scores, void* ws,
                size_t ws_bytes, void* stream);
