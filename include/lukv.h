@@ -229,6 +229,16 @@ LUKV_API int lukv_compress_ragged(const lukv_params_t* params, const int32_t* ct
                                   const void* k, const void* v, const float* curves, const int64_t* budgets_in,
                                   void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets, int32_t* offsets,
                                   int64_t rows_cap, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+/*
+ * Stages (c) and (d) for such a batch, for callers that bring their own budgets -- with lukv_profile_budgets_ragged
+ * and lukv_score_ragged this is the paper's deployment mode (Sec. 4.3 "Online Execution") on sequences of different
+ * lengths.  Arguments as lukv_select_gather; scores [S][N][T-w] with the first n_q entries of a row read;
+ * 0 <= budgets[u] <= n_q; head u of sequence q keeps its window rows n_q .. ctx_lens[q]-1.
+ */
+LUKV_API int lukv_select_gather_ragged(const lukv_params_t* params, const int32_t* ctx_lens, const float* scores,
+                                       const int32_t* budgets, const int32_t* offsets, const void* k, const void* v,
+                                       void* k_out, void* v_out, int32_t* kept_idx, int64_t rows_cap, void* ws,
+                                       size_t ws_bytes, void* stream);
 
 /*
  * Profiling variant of lukv_compress (the paper has no counterpart): same arguments and
@@ -317,6 +327,14 @@ LUKV_API int lukv_profile_build(const lukv_params_t* calib, const float* curves,
 LUKV_API int lukv_profile_budgets(const lukv_params_t* params, const float* profile, const float* ratios,
                                   int32_t n_ratios, const float* sigma, int32_t* budgets, int32_t* offsets,
                                   void* stream);
+/*
+ * The same for sequences of different context lengths (see lukv_compress_ragged for ctx_lens): head h of sequence
+ * q gets b = floor((1-r)*n_q), n_q = ctx_lens[q] - w, raised to ceil(min_keep*n_q); the result equals one
+ * single-sequence call per sequence, concatenated (offsets running over all sequences).
+ */
+LUKV_API int lukv_profile_budgets_ragged(const lukv_params_t* params, const int32_t* ctx_lens, const float* profile,
+                                         const float* ratios, int32_t n_ratios, const float* sigma,
+                                         int32_t* budgets, int32_t* offsets, void* stream);
 
 /*
  * Utility-versus-budget curves of the proxy metric (Sec. 3.2: M^pi(k) is the set of the first k

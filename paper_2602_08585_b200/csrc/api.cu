@@ -303,12 +303,14 @@ int lukv_allocate(const lukv_params_t* params, const float* curves, const int64_
   return LUKV_OK;
 }
 
-int lukv_select_gather(const lukv_params_t* params, const float* scores, const int32_t* budgets, const int32_t* offsets,
-                       const void* k, const void* v, void* k_out, void* v_out, int32_t* kept_idx, int64_t rows_cap,
-                       void* ws, size_t ws_bytes, void* stream) {
+static int select_gather_impl(const lukv_params_t* params, const int32_t* ctx_lens, bool ragged, const float* scores,
+                              const int32_t* budgets, const int32_t* offsets, const void* k, const void* v, void* k_out,
+                              void* v_out, int32_t* kept_idx, int64_t rows_cap, void* ws, size_t ws_bytes,
+                              void* stream) {
   Dims dm;
   int rc = make_dims(params, &dm);
   if (rc != LUKV_OK) return rc;
+  if (ragged && (rc = attach_seq_lens(&dm, ctx_lens)) != LUKV_OK) return rc;
   if (!scores || !budgets || !offsets || !k || !v || !k_out || !v_out || !kept_idx || rows_cap < 0 || !aligned16(k) ||
       !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
     return LUKV_ERR_INVALID_ARG;
@@ -322,6 +324,21 @@ int lukv_select_gather(const lukv_params_t* params, const float* scores, const i
     return LUKV_ERR_CUDA;
   g_last_launches = lc.launches;
   return LUKV_OK;
+}
+
+int lukv_select_gather(const lukv_params_t* params, const float* scores, const int32_t* budgets, const int32_t* offsets,
+                       const void* k, const void* v, void* k_out, void* v_out, int32_t* kept_idx, int64_t rows_cap,
+                       void* ws, size_t ws_bytes, void* stream) {
+  return select_gather_impl(params, nullptr, false, scores, budgets, offsets, k, v, k_out, v_out, kept_idx, rows_cap, ws,
+                            ws_bytes, stream);
+}
+
+int lukv_select_gather_ragged(const lukv_params_t* params, const int32_t* ctx_lens, const float* scores,
+                              const int32_t* budgets, const int32_t* offsets, const void* k, const void* v, void* k_out,
+                              void* v_out, int32_t* kept_idx, int64_t rows_cap, void* ws, size_t ws_bytes,
+                              void* stream) {
+  return select_gather_impl(params, ctx_lens, true, scores, budgets, offsets, k, v, k_out, v_out, kept_idx, rows_cap, ws,
+                            ws_bytes, stream);
 }
 
 int lukv_compress(const lukv_params_t* params, const void* q_win, const void* k, const void* v, const float* curves,
@@ -519,11 +536,13 @@ int lukv_profile_build(const lukv_params_t* calib, const float* curves, int32_t 
   return LUKV_OK;
 }
 
-int lukv_profile_budgets(const lukv_params_t* params, const float* profile, const float* ratios, int32_t n_ratios,
-                         const float* sigma, int32_t* budgets, int32_t* offsets, void* stream) {
+static int profile_budgets_impl(const lukv_params_t* params, const int32_t* ctx_lens, bool ragged, const float* profile,
+                                const float* ratios, int32_t n_ratios, const float* sigma, int32_t* budgets,
+                                int32_t* offsets, void* stream) {
   Dims dm;
   int rc = make_dims(params, &dm);
   if (rc != LUKV_OK) return rc;
+  if (ragged && (rc = attach_seq_lens(&dm, ctx_lens)) != LUKV_OK) return rc;
   if (!profile || !ratios || !sigma || !budgets || !offsets || n_ratios < 1) return LUKV_ERR_INVALID_ARG;
   for (int j = 0; j + 1 < n_ratios; ++j)
     if (!(ratios[j] < ratios[j + 1])) return LUKV_ERR_INVALID_ARG;
@@ -549,11 +568,22 @@ int lukv_profile_budgets(const lukv_params_t* params, const float* profile, cons
   LaunchCtx lc;
   lc.st = (cudaStream_t)stream;
   const cudaError_t e =
-      launch_profile_budgets(profile, row_lo, row_hi, frac, dm.S, dm.N, dm.n, dm.w, dm.floor_tok, budgets, offsets, lc);
+      launch_profile_budgets(profile, row_lo, row_hi, frac, dm, budgets, offsets, lc);
   free(rows);
   if (e != cudaSuccess) return LUKV_ERR_CUDA;
   g_last_launches = lc.launches;
   return LUKV_OK;
+}
+
+int lukv_profile_budgets(const lukv_params_t* params, const float* profile, const float* ratios, int32_t n_ratios,
+                         const float* sigma, int32_t* budgets, int32_t* offsets, void* stream) {
+  return profile_budgets_impl(params, nullptr, false, profile, ratios, n_ratios, sigma, budgets, offsets, stream);
+}
+
+int lukv_profile_budgets_ragged(const lukv_params_t* params, const int32_t* ctx_lens, const float* profile,
+                                const float* ratios, int32_t n_ratios, const float* sigma, int32_t* budgets,
+                                int32_t* offsets, void* stream) {
+  return profile_budgets_impl(params, ctx_lens, true, profile, ratios, n_ratios, sigma, budgets, offsets, stream);
 }
 
 int lukv_build_curves(const lukv_params_t* params, const float* scores, const float* importance, float* curves,

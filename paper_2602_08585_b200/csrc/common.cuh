@@ -124,8 +124,7 @@ cudaError_t launch_profile_mean(const int32_t* budgets, float* profile, int n_qu
                                 LaunchCtx& lc);
 constexpr int kLookupSeqPerLaunch = 32;
 cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, const int* row_hi, const double* frac,
-                                   int S, int N, int n, int w, int floor_tok, int32_t* budgets, int32_t* offsets,
-                                   LaunchCtx& lc);
+                                   const Dims& dm, int32_t* budgets, int32_t* offsets, LaunchCtx& lc);
 // Curves of a proxy ranking: scores, importance [heads][n] -> curves [heads][P].
 size_t curves_smem_bytes(int n, int P);
 cudaError_t launch_build_curves(const Dims& dm, const float* scores, const float* importance, float* curves,

@@ -32,15 +32,18 @@ struct LookupArgs {
   int row_lo[kLookupSeqPerLaunch];   // grid row at or below the target ratio
   int row_hi[kLookupSeqPerLaunch];   // the next row (== row_lo at the last grid point)
   double frac[kLookupSeqPerLaunch];  // position of the target between the two rows, in [0,1)
+  int n[kLookupSeqPerLaunch];        // rankable positions of the sequence
+  int floor_tok[kLookupSeqPerLaunch];  // its minimum retention in tokens
   int seq0;
 };
 
 // blockIdx.y = sequence of this launch, x covers the heads.
-__global__ void profile_budget_kernel(const float* __restrict__ profile, LookupArgs args, int N, int n,
-                                      int floor_tok, int32_t* __restrict__ budgets) {
+__global__ void profile_budget_kernel(const float* __restrict__ profile, LookupArgs args, int N,
+                                      int32_t* __restrict__ budgets) {
   const int hid = blockIdx.x * kProfileThreads + threadIdx.x;
   if (hid >= N) return;
   const int i = blockIdx.y;
+  const int n = args.n[i], floor_tok = args.floor_tok[i];
   const double r0 = (double)profile[(size_t)args.row_lo[i] * N + hid];
   const double r1 = (double)profile[(size_t)args.row_hi[i] * N + hid];
   const double r = __dadd_rn(r0, __dmul_rn(__dsub_rn(r1, r0), args.frac[i]));
@@ -90,8 +93,8 @@ cudaError_t launch_profile_mean(const int32_t* budgets, float* profile, int n_qu
 }
 
 cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, const int* row_hi, const double* frac,
-                                   int S, int N, int n, int w, int floor_tok, int32_t* budgets, int32_t* offsets,
-                                   LaunchCtx& lc) {
+                                   const Dims& dm, int32_t* budgets, int32_t* offsets, LaunchCtx& lc) {
+  const int S = dm.S, N = dm.N, w = dm.w;
   for (int q0 = 0; q0 < S; q0 += kLookupSeqPerLaunch) {
     LookupArgs args;
     const int cnt = S - q0 < kLookupSeqPerLaunch ? S - q0 : kLookupSeqPerLaunch;
@@ -99,10 +102,12 @@ cudaError_t launch_profile_budgets(const float* profile, const int* row_lo, cons
       args.row_lo[i] = i < cnt ? row_lo[q0 + i] : 0;
       args.row_hi[i] = i < cnt ? row_hi[q0 + i] : 0;
       args.frac[i] = i < cnt ? frac[q0 + i] : 0.0;
+      args.n[i] = i < cnt ? seq_rankable(dm, q0 + i) : 0;
+      args.floor_tok[i] = i < cnt ? seq_floor_tokens(dm, q0 + i) : 0;
     }
     args.seq0 = q0;
     profile_budget_kernel<<<dim3((N + kProfileThreads - 1) / kProfileThreads, cnt), kProfileThreads, 0, lc.st>>>(
-        profile, args, N, n, floor_tok, budgets);
+        profile, args, N, budgets);
     lc.mark("profile_budget");
   }
   offsets_scan_kernel<<<1, kScanThreads, 0, lc.st>>>(budgets, offsets, S * N, w);

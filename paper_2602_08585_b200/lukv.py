@@ -25,7 +25,8 @@ EXPORTS = ("lukv_workspace_bytes", "lukv_score", "lukv_allocate", "lukv_select_g
            "lukv_strerror", "lukv_last_launch_count", "lukv_compress_profile", "lukv_allocate_static",
            "lukv_profile_workspace_bytes", "lukv_profile_build", "lukv_profile_budgets", "lukv_build_curves", "lukv_exact_workspace_bytes",
            "lukv_exact_allocate", "lukv_importance_workspace_bytes", "lukv_oracle_importance", "lukv_score_ragged",
-           "lukv_compress_ragged", "lukv_score_keydiff")
+           "lukv_compress_ragged", "lukv_score_keydiff", "lukv_select_gather_ragged",
+           "lukv_profile_budgets_ragged")
 
 
 class Params(ctypes.Structure):
@@ -89,6 +90,8 @@ def lib() -> ctypes.CDLL:
         L.lukv_score_ragged.argtypes = [pp, vp, vp, vp, vp, vp, sz, vp]
         L.lukv_score_keydiff.argtypes = [pp, vp, vp, vp, vp, sz, vp]
         L.lukv_compress_ragged.argtypes = [pp, vp] + L.lukv_compress.argtypes[1:]
+        L.lukv_select_gather_ragged.argtypes = [pp, vp] + L.lukv_select_gather.argtypes[1:]
+        L.lukv_profile_budgets_ragged.argtypes = [pp, vp] + L.lukv_profile_budgets.argtypes[1:]
         L.lukv_strerror.argtypes = [ctypes.c_int]
         L.lukv_strerror.restype = ctypes.c_char_p
         for name in EXPORTS[:5] + EXPORTS[6:]:
@@ -200,6 +203,18 @@ def lukv_profile_budgets(params: Params, profile, ratios, sigma, budgets, offset
     return _check(rc, "lukv_profile_budgets", check)
 
 
+def lukv_profile_budgets_ragged(params: Params, ctx_lens, profile, ratios, sigma, budgets, offsets, stream=None,
+                                check: bool = True) -> int:
+    """lukv_profile_budgets for sequences of different lengths: ctx_lens [S] host ints."""
+    r, sg, lens = _host_f32(ratios), _host_f32(sigma), _host_lens(ctx_lens)
+    if sg.shape[0] != params.batch:
+        raise ValueError("one target ratio per sequence")
+    rc = lib().lukv_profile_budgets_ragged(ctypes.byref(params), lens.ctypes.data, _ptr(profile), r.ctypes.data,
+                                           int(r.shape[0]), sg.ctypes.data, _ptr(budgets), _ptr(offsets),
+                                           _stream(stream))
+    return _check(rc, "lukv_profile_budgets_ragged", check)
+
+
 def lukv_build_curves(params: Params, scores, importance, curves, stream=None, check: bool = True) -> int:
     """Curves of the proxy ranking: scores, importance [S][N][n] -> curves [S][N][P] (all device)."""
     rc = lib().lukv_build_curves(ctypes.byref(params), _ptr(scores), _ptr(importance), _ptr(curves), _stream(stream))
@@ -248,6 +263,17 @@ def lukv_select_gather(params: Params, scores, budgets, offsets, k, v, k_out, v_
                                   _ptr(k_out), _ptr(v_out), _ptr(kept_idx), int(rows_cap), _ptr(ws),
                                   0 if ws is None else ws.numel() * ws.element_size(), _stream(stream))
     return _check(rc, "lukv_select_gather", check)
+
+
+def lukv_select_gather_ragged(params: Params, ctx_lens, scores, budgets, offsets, k, v, k_out, v_out, kept_idx,
+                              rows_cap: int, ws, stream=None, check: bool = True) -> int:
+    """lukv_select_gather for sequences of different lengths: ctx_lens [S] host ints."""
+    lens = _host_lens(ctx_lens)
+    rc = lib().lukv_select_gather_ragged(ctypes.byref(params), lens.ctypes.data, _ptr(scores), _ptr(budgets),
+                                         _ptr(offsets), _ptr(k), _ptr(v), _ptr(k_out), _ptr(v_out), _ptr(kept_idx),
+                                         int(rows_cap), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                         _stream(stream))
+    return _check(rc, "lukv_select_gather_ragged", check)
 
 
 def lukv_compress(params: Params, q_win, k, v, curves, budgets_in, k_out, v_out, kept_idx, budgets, offsets,

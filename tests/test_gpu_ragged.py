@@ -97,6 +97,61 @@ def test_equal_lengths_match_the_batched_call():
     assert torch.equal(a.k_out.view(torch.int16), b.k_out.view(torch.int16))
 
 
+def test_online_mode_on_sequences_of_different_lengths(oracle):
+    """The deployment mode of Sec. 4.3 (lookup and budgeting -> scoring -> eviction) on a ragged batch:
+    lukv_profile_budgets_ragged, lukv_score_ragged, lukv_select_gather_ragged against one single-sequence oracle run
+    per sequence.  Budgets and offsets exact; selection and gather exact on the oracle's scores."""
+    S, L, H, G, d, T, w, kp = 3, 2, 2, 4, 128, 2048, 32, 7
+    lens, N, R = [2048, 1280, 700], 4, 9
+    g = torch.Generator().manual_seed(12)
+    q = torch.randn((S, L, H * G, w, d), generator=g).to(torch.bfloat16)
+    k = torch.randn((S, L, H, T, d), generator=g).to(torch.bfloat16)
+    v = torch.randn((S, L, H, T, d), generator=g).to(torch.bfloat16)
+    rng = np.random.default_rng(12)
+    ratios = np.linspace(0.1, 0.9, R).astype(np.float32)
+    profile = np.sort(rng.random((R, N)).astype(np.float32), axis=0)        # per head non-decreasing in the ratio
+    sigma = np.asarray([0.3, 0.55, 0.9], np.float32)                         # a grid point, between two, the last
+    p = lukv.make_params(S, L, H, G, d, T, w, kp, torch.bfloat16, 2, n_sink=4, min_keep=0.02)
+    budgets = torch.full((S, N), -1, dtype=torch.int32, device="cuda")
+    offsets = torch.full((S * N + 1,), -1, dtype=torch.int32, device="cuda")
+    lukv.lukv_profile_budgets_ragged(p, lens, torch.from_numpy(profile).cuda(), ratios, sigma, budgets, offsets)
+    torch.cuda.synchronize()
+    ref_b = np.concatenate([oracle.profile_budgets(profile, ratios, lens[s], w, sigma[s:s + 1], min_keep=0.02)[0]
+                            for s in range(S)])
+    ref_o = np.concatenate([[0], np.cumsum(ref_b.reshape(-1) + w)]).astype(np.int32)
+    np.testing.assert_array_equal(budgets.cpu().numpy(), ref_b)
+    np.testing.assert_array_equal(offsets.cpu().numpy(), ref_o)
+    for s in range(S):
+        assert ref_b[s].min() >= int(np.ceil(np.float32(0.02) * (lens[s] - w)))
+    # scores of the ragged call, then eviction on the oracle's scores (so that near-ties cannot reorder positions)
+    ws = lukv.alloc_workspace(p)
+    scores = torch.zeros((S, N, T - w), dtype=torch.float32, device="cuda")
+    lukv.lukv_score_ragged(p, lens, q.cuda(), k.cuda(), scores, ws)
+    ref_scores = np.zeros((S, N, T - w), np.float32)
+    for s, Ts in enumerate(lens):
+        ref_scores[s, :, :Ts - w] = oracle.score(bits(q[s:s + 1]), bits(k[s:s + 1, :, :, :Ts].contiguous()), G, kp)[0]
+    torch.cuda.synchronize()
+    for s, Ts in enumerate(lens):
+        assert_scores_close(scores.cpu().numpy()[s, :, :Ts - w], ref_scores[s, :, :Ts - w])
+    rows = int(ref_o[-1])
+    k_out = torch.zeros((rows, d), dtype=torch.bfloat16, device="cuda")
+    v_out = torch.zeros((rows, d), dtype=torch.bfloat16, device="cuda")
+    kept = torch.full((rows,), -1, dtype=torch.int32, device="cuda")
+    lukv.lukv_select_gather_ragged(p, lens, torch.from_numpy(ref_scores).cuda(), budgets, offsets, k.cuda(), v.cuda(),
+                                   k_out, v_out, kept, rows, ws)
+    torch.cuda.synchronize()
+    kept, ko, vo = kept.cpu().numpy(), bits(k_out), bits(v_out)
+    for s, Ts in enumerate(lens):
+        r0 = ref_o[s * N]
+        rk, rv, rkept = oracle.select_gather(ref_scores[s, :, :Ts - w], ref_b[s], ref_o[s * N:(s + 1) * N + 1] - r0,
+                                             bits(k[s, :, :, :Ts].contiguous()).reshape(N, Ts, d),
+                                             bits(v[s, :, :, :Ts].contiguous()).reshape(N, Ts, d), w, n_sink=4)
+        r1 = ref_o[(s + 1) * N]
+        np.testing.assert_array_equal(kept[r0:r1], rkept)
+        np.testing.assert_array_equal(ko[r0:r1], rk)
+        np.testing.assert_array_equal(vo[r0:r1], rv)
+
+
 def test_ragged_argument_errors():
     p = lukv.make_params(2, 1, 2, 2, 64, 256, 8, 3, "bf16", 17)
     f = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
