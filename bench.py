@@ -645,7 +645,7 @@ def run_profile_path(args):
                            "frac_by_design": (keydiff_k_bytes + keydiff_bytes) / (keydiff_ms * 1e-3) / 1e9
                                              / measured_peak()[0]},
         "build_curves": {"ms_per_call": curves_ms, "queries": Mq, "heads": wl.N, "positions": Tc - wl.w,
-                         "compares": float(Mq) * wl.N * (Tc - wl.w) ** 2},
+                         "algorithmic_bytes": Mq * wl.N * ((Tc - wl.w) * 8 + (Tc + 1) * 4)},
         "online_mode": {"metric": METRIC, "value": wl.S * wl.T / (online_ms * 1e-3), "unit": UNIT,
                         "ms_per_step": online_ms, "packed_rows": rows, "launches_per_step": sum(counts),
                         "path_bytes_per_step": wl.S * wl.N * wl.T * wl.d * es + 2 * rows * wl.d * es},

@@ -50,6 +50,11 @@ def test_calibration_size(oracle):
     assert (np.diff(got.astype(np.float64), axis=-1) >= 0).all()
 
 
+def test_beyond_the_sorting_kernel(oracle):
+    # more than 16384 positions: ranks by counting instead of the shared-memory sort
+    _case(oracle, 1, 1, 2, 20000, 32, 126, n_sink=4, seed=6, ties=True)
+
+
 def test_too_long_contexts_are_refused():
     p = lukv.make_params(1, 1, 1, 1, 64, 32768, 32, 1, "fp32", 257)
     f = torch.empty(1, device="cuda")
