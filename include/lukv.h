@@ -201,7 +201,8 @@ LUKV_API int lukv_select_gather(const lukv_params_t* params, const float* scores
  * after earlier work on `stream` and before later work on it.  Host threads may call
  * concurrently on one device (each with its own workspace and outputs): the call holds a
  * per-device lock while it enqueues on the auxiliary stream, so such calls enqueue one after
- * the other.
+ * the other.  The call only enqueues (kernels, memsets, the event pair), so it may be captured into a CUDA
+ * graph once the auxiliary stream exists (after one plain call on the device).
  */
 LUKV_API int lukv_compress(const lukv_params_t* params, const void* q_win, const void* k, const void* v,
                   const float* curves, const int64_t* budgets_in, void* k_out, void* v_out, int32_t* kept_idx,

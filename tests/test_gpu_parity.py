@@ -330,3 +330,35 @@ print("ok")
     env = dict(os.environ, LUKV_QUADS="3")
     out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
+
+
+def test_compress_can_be_captured_in_a_cuda_graph():
+    """The whole call only enqueues (kernels, two small memsets, an event pair on the auxiliary stream), so a caller
+    may capture it into a CUDA graph; replays give the same bytes as the plain call."""
+    wl = synth.scaled(synth.CONFIGS["llama8b_1layer_8k"], H=4, T=4096, P=65)
+    q, k, v = synth.gen_tensors(wl, "cuda")
+    curves = torch.from_numpy(synth.gen_curves(wl)).cuda()
+    Bs = wl.budgets()
+    p = params_of(wl)
+    ws = lukv.alloc_workspace(p)
+    plain, out = lukv.Outputs(p, Bs), lukv.Outputs(p, Bs)
+
+    def call(o):
+        lukv.lukv_compress(p, q, k, v, curves, Bs, o.k_out, o.v_out, o.kept_idx, o.budgets, o.offsets, o.rows,
+                           o.dev_status, ws)
+
+    call(plain)
+    torch.cuda.synchronize()
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            call(out)
+    for _ in range(3):
+        out.kept_idx.fill_(-1)
+        out.k_out.zero_()
+        graph.replay()
+    torch.cuda.synchronize()
+    assert int(out.dev_status.item()) == 0
+    assert torch.equal(out.budgets, plain.budgets) and torch.equal(out.kept_idx, plain.kept_idx)
+    assert torch.equal(out.k_out.view(torch.int16), plain.k_out.view(torch.int16))
+    assert torch.equal(out.v_out.view(torch.int16), plain.v_out.view(torch.int16))
