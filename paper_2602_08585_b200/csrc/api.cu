@@ -172,8 +172,9 @@ static int run_compress(const Dims& dm, const void* q_win, const void* k, const 
                         bool overlap) {
   if (dev_status && cudaMemsetAsync(dev_status, 0, sizeof(int32_t), lc.st) != cudaSuccess) return LUKV_ERR_CUDA;
   const bool tc = score_tc_supported(dm) && !force_simt();
-  // the persistent scorers (tensor-core, KeyDiff) leave one SM to the allocation kernels of the auxiliary stream
-  SideStream* side = (overlap && (tc || dm.keydiff)) ? side_stream() : nullptr;
+  // the persistent scorers (tensor-core, KeyDiff) leave one SM to the allocation kernels of the auxiliary stream;
+  // the FP32-pipe scorer's ordinary grids simply share the SMs with them
+  SideStream* side = overlap ? side_stream() : nullptr;
   int rc = LUKV_OK;
   if (side) {
     std::lock_guard<std::mutex> in_use(side->use);
@@ -186,9 +187,12 @@ static int run_compress(const Dims& dm, const void* q_win, const void* k, const 
     lc.launches += ls.launches;
     if (rc == LUKV_OK && dm.keydiff) {
       if (launch_keydiff(dm, k, w.pooled, w.stats, dev_status, 1, lc) != cudaSuccess) rc = LUKV_ERR_CUDA;
-    } else if (rc == LUKV_OK && (launch_score_tc(dm, q_win, k, w, dev_status, all_heads(dm), true, 1, lc) != cudaSuccess ||
-                                 launch_pool(dm, w.raw, w.pooled, all_heads(dm), lc) != cudaSuccess)) {
-      rc = LUKV_ERR_CUDA;
+    } else if (rc == LUKV_OK && tc) {
+      if (launch_score_tc(dm, q_win, k, w, dev_status, all_heads(dm), true, 1, lc) != cudaSuccess ||
+          launch_pool(dm, w.raw, w.pooled, all_heads(dm), lc) != cudaSuccess)
+        rc = LUKV_ERR_CUDA;
+    } else if (rc == LUKV_OK) {
+      if (run_score(dm, q_win, k, w, w.pooled, dev_status, lc) != cudaSuccess) rc = LUKV_ERR_CUDA;
     }
     // join even after a failure: the caller's stream must not run ahead of work already enqueued
     if (cudaStreamWaitEvent(lc.st, side->join, 0) != cudaSuccess) rc = LUKV_ERR_CUDA;
