@@ -325,13 +325,13 @@ cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* bu
   const int hps = dm.seq_T ? dm.N : 0;
   if (dm.seq_T)
     for (int q = 0; q < dm.S; ++q) sl.T[q] = dm.seq_T[q];
-  // Keys per thread (in registers) and CTAs per head.  Up to 32768 positions: one CTA with 2, 8 or 32 keys per
+  // Keys per thread (in registers) and CTAs per head.  Up to 32768 positions: one CTA with 2, 8, 16 or 32 keys per
   // thread (a cluster's barriers cost more than they save there).  Up to 262144: the smallest cluster (2, 4 or 8
   // CTAs) that covers the head with 32 keys per thread; small clusters are placed and synchronised faster than large
   // ones.  Beyond: one CTA that re-reads its keys from memory in every round.
   int ept = 0, csize = 1;
   if (n <= kSelThreads * 32) {
-    ept = n <= kSelThreads * 2 ? 2 : n <= kSelThreads * 8 ? 8 : 32;
+    ept = n <= kSelThreads * 2 ? 2 : n <= kSelThreads * 8 ? 8 : n <= kSelThreads * 16 ? 16 : 32;
   } else {
     for (int c : {2, 4, 8})
       if (!ept && (long long)c * kSelThreads * 32 >= n) ept = 32, csize = c;
@@ -342,7 +342,8 @@ cudaError_t launch_select(const Dims& dm, const float* scores, const int32_t* bu
     select_kernel<0, false><<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, span,
                                                           hr.h0, dm.n_sink, sl, hps);
   } else if (csize == 1) {
-    auto kern = ept == 2 ? select_kernel<2, false> : ept == 8 ? select_kernel<8, false> : select_kernel<32, false>;
+    auto kern = ept == 2 ? select_kernel<2, false> : ept == 8 ? select_kernel<8, false>
+                         : ept == 16 ? select_kernel<16, false> : select_kernel<32, false>;
     kern<<<grid, kSelThreads, 0, st>>>(scores, budgets, offsets, kept_idx, rows_cap, n, dm.w, 0, hr.h0, dm.n_sink, sl,
                                        hps);
   } else {
