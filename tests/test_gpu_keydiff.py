@@ -190,6 +190,28 @@ def test_keydiff_whole_path_by_flag(oracle, dtype):
     np.testing.assert_allclose(scores.cpu().numpy(), ref_scores, rtol=0, atol=ATOL)
 
 
+def test_keydiff_flag_in_the_profiling_call():
+    """lukv_compress_profile with the flag runs the same kernels one after the other: same bytes, and the timeline
+    names the KeyDiff kernel instead of the attention scorer and the pooling."""
+    wl = synth.scaled(synth.CONFIGS["llama8b_1layer_8k"], H=3, T=2048, w=1, kp=1, P=65)
+    _, k, v = synth.gen_tensors(wl, "cuda")
+    curves = torch.from_numpy(synth.gen_curves(wl)).cuda()
+    Bs = [int(0.3 * wl.N * (wl.T - 1))]
+    p = lukv.make_params(wl.S, wl.L, wl.H, wl.G, wl.d, wl.T, wl.w, wl.kp, wl.dtype, wl.P, flags=lukv.FLAG_KEYDIFF)
+    ws = lukv.alloc_workspace(p)
+    a, b = lukv.Outputs(p, Bs), lukv.Outputs(p, Bs)
+    lukv.lukv_compress(p, None, k, v, curves, Bs, a.k_out, a.v_out, a.kept_idx, a.budgets, a.offsets, a.rows,
+                       a.dev_status, ws)
+    times = lukv.lukv_compress_profile(p, None, k, v, curves, Bs, b.k_out, b.v_out, b.kept_idx, b.budgets, b.offsets,
+                                       b.rows, b.dev_status, ws)
+    torch.cuda.synchronize()
+    names = [name for name, _ in times]
+    assert "keydiff" in names and not any("score" in name or "pool" in name for name in names)
+    assert all(ms >= 0.0 for _, ms in times)
+    assert torch.equal(a.kept_idx, b.kept_idx) and torch.equal(a.budgets, b.budgets)
+    assert torch.equal(a.k_out.view(torch.int16), b.k_out.view(torch.int16))
+
+
 def test_keydiff_flag_argument_errors():
     f = torch.empty(4096, dtype=torch.uint8, device="cuda")
     pooled = lukv.make_params(1, 1, 2, 1, 64, 256, 1, 7, "bf16", 2, flags=lukv.FLAG_KEYDIFF)   # the metric is not pooled
