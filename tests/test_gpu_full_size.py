@@ -152,3 +152,32 @@ def test_repeated_calls_are_bit_identical():
             scores.fill_(-1.0)
             lukv.lukv_score(p, q, k, scores, ws)
             assert torch.equal(scores, scores0), rep
+
+
+def test_keydiff_full_size_sampled_heads(oracle):
+    """KeyDiff scores at the headline size (256 heads x 32768 keys, the launch bench.py times): 16 sampled heads
+    element by element against the oracle; every score is a cosine; two calls give the same bits."""
+    wl = synth.CONFIGS["llama8b_32k"]
+    _, k, _ = synth.gen_tensors(wl, "cuda")
+    p = lukv.make_params(wl.S, wl.L, wl.H, 1, wl.d, wl.T, 1, 1, wl.dtype, 2)
+    ws = lukv.alloc_workspace(p)
+    n = wl.T - 1
+    scores = torch.full((wl.S, wl.N, n), 7.0, dtype=torch.float32, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    lukv.lukv_score_keydiff(p, k, scores, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    first = scores.clone()
+    assert float(scores.abs().max()) <= 1.0 + 1e-5
+    scores.fill_(7.0)
+    lukv.lukv_score_keydiff(p, k, scores, ws, status)
+    torch.cuda.synchronize()
+    assert torch.equal(scores, first)
+    heads = wl.S * wl.N
+    rng = np.random.default_rng(wl.seed + 1)
+    sample = sorted(set(int(x) for x in rng.integers(0, heads, size=14)) | {0, heads - 1})
+    kh = k.reshape(heads, wl.T, wl.d)
+    got = scores.reshape(heads, n)
+    for u in sample:
+        ref = oracle.keydiff(bits(kh[u].cpu()).reshape(1, 1, 1, wl.T, wl.d), 1).reshape(n)
+        np.testing.assert_allclose(got[u].cpu().numpy(), ref, rtol=0, atol=2e-5)
