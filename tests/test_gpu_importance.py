@@ -76,6 +76,31 @@ def test_value_norms_tensor_core_against_fp32_pipes(monkeypatch):
     np.testing.assert_allclose(tc, simt, rtol=2e-5, atol=1e-30)
 
 
+def test_importance_at_the_benchmark_size_sampled_heads(oracle):
+    """The size bench.py times (one calibration query of 4000 tokens, 256 KV heads x 4 query heads, 64 decode steps,
+    model width 4096; the value norms run on the tensor cores over 1024 work items): two sampled heads against the
+    oracle, without the per-layer normalisation (which would need every head of the layer)."""
+    S, L, H, G, d, T, w, Kmax, Dm = 1, 32, 8, 4, 128, 4000, 32, 64, 4096
+    g = torch.Generator(device="cuda").manual_seed(3)
+    dt = torch.bfloat16
+    q = torch.randn((S, L, H * G, Kmax, d), generator=g, device="cuda").to(dt)
+    k = torch.randn((S, L, H, T, d), generator=g, device="cuda").to(dt)
+    v = torch.randn((S, L, H, T, d), generator=g, device="cuda").to(dt)
+    kd = torch.randn((S, L, H, Kmax, d), generator=g, device="cuda").to(dt)
+    wo = (torch.randn((L, H * G, d, Dm), generator=g, device="cuda") / d ** 0.5).to(dt)
+    p = lukv.make_params(S, L, H, G, d, T, w, 1, dt, 2)
+    ws = torch.empty(lukv.lukv_importance_workspace_bytes(p, Kmax), dtype=torch.uint8, device="cuda")
+    out = torch.full((S, L * H, T - w), -7.0, dtype=torch.float32, device="cuda")
+    lukv.lukv_oracle_importance(p, Kmax, Dm, q, k, v, kd, wo, False, out, ws)
+    torch.cuda.synchronize()
+    for layer, h in [(0, 0), (19, 5)]:
+        sub = lambda t, lo, hi: bits(t[:, layer:layer + 1, lo:hi].contiguous().cpu())
+        ref = oracle.importance(sub(q, h * G, (h + 1) * G), sub(k, h, h + 1), sub(v, h, h + 1),
+                                bits(wo[layer:layer + 1, h * G:(h + 1) * G].contiguous().cpu()), G, w,
+                                k_dec=sub(kd, h, h + 1), normalize=False)
+        _close(out[:, layer * H + h].cpu().numpy().reshape(ref.shape), ref)
+
+
 def test_importance_argument_errors():
     p = lukv.make_params(1, 1, 2, 2, 64, 256, 8, 1, "bf16", 2)
     f = torch.empty(1024, dtype=torch.uint8, device="cuda")
